@@ -1,0 +1,245 @@
+/*
+ * cdma.h -- C ABI of the compressing-DMA (cDMA) zero-value-compression library
+ *           for NVIDIA B200 (sm_100a).
+ *
+ * The paper proposes a memory copy that compresses activation maps on their
+ * way from GPU memory to host memory and expands them on the way back, and
+ * that reports the compressed size when the copy completes (Section V-D,
+ * "Software Interface": cudaMemcpyCompressed).  This library provides that
+ * operation in software: the codec runs as CUDA kernels on the SMs, the copy
+ * over the host link is a plain cudaMemcpyAsync of the compressed bytes.
+ *
+ * Stream format (Section V-A, "Zero-value compression"):
+ *   elements are taken 32 at a time in memory order (a "window").  A window's
+ *   record is a 32-bit mask, least-significant byte first, bit i set when
+ *   element i of the window is non-zero, followed by the window's non-zero
+ *   elements in ascending order, bytes unchanged.  "Non-zero" is a test of
+ *   the element's bit pattern (Section V-B: words are compared to zero), so
+ *   -0.0, NaNs, denormals and infinities are kept.  The payload is the
+ *   concatenation of all records with no header and no padding; its size is
+ *   4*ceil(n/32) + s*nnz bytes for n elements of s bytes of which nnz are
+ *   non-zero.  A short last window has zero bits for the missing elements.
+ *   For 2-byte elements the window is still 32 elements with a 32-bit mask.
+ *
+ * Framing for parallel decoding (outside the payload): an offset table of
+ *   ceil(n/1024)+1 little-endian uint64.  Entry k is the payload offset of
+ *   the record of window 32k ("chunk" k = 1024 elements, the 4 KB block of the
+ *   paper's compression study, Fig. 11 caption); the last entry equals the
+ *   payload size.
+ *
+ * Conventions
+ *   - "d_" pointers are device memory of the current CUDA device, "h_"
+ *     pointers are host memory.  Streams are passed as void* holding a
+ *     cudaStream_t (NULL = the legacy default stream).
+ *   - The caller owns every buffer passed in; the codec calls allocate
+ *     nothing.  A cdma_ctx owns its pinned host pool, its device staging and
+ *     its side stream.
+ *   - Dense tensors and compressed buffers must start on a 16-byte boundary
+ *     and must not overlap each other.  The tensor must be dense in its
+ *     physical layout; the layout argument is a tag that is validated and
+ *     recorded but does not change the bytes: the codec compresses memory
+ *     order (Section V-A: ZVC is insensitive to the layout).
+ *   - Functions returning int64_t return a byte count >= 0, or -status on
+ *     failure.  Functions returning int return a status (0 = success).
+ *     Nothing aborts, throws or traps; device-side failures (capacity
+ *     overflow, malformed stream, a wait that ran out) are written to a
+ *     status word and come back as a negative return.
+ *   - A call never writes beyond dst_capacity / n elements, whatever the
+ *     input holds.  Bytes of the destination between the payload's end and
+ *     dst_capacity, and the contents of workspaces, are unspecified.
+ *   - Not thread-safe per context or per workspace: two calls that share a
+ *     workspace (or a context) must not overlap in time.
+ */
+#ifndef CDMA_H_
+#define CDMA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes; negative returns are the negated code */
+enum {
+    CDMA_OK = 0,
+    CDMA_ERR_INVALID_ARG = 1,        /* null pointer, overlap, size mismatch            */
+    CDMA_ERR_UNSUPPORTED_DTYPE = 2,
+    CDMA_ERR_UNSUPPORTED_LAYOUT = 3,
+    CDMA_ERR_ALIGNMENT = 4,          /* a buffer is not 16-byte aligned                 */
+    CDMA_ERR_BUFFER_TOO_SMALL = 5,   /* payload, table, workspace or pool too small     */
+    CDMA_ERR_CORRUPT_STREAM = 6,     /* table or payload fails validation in decompress */
+    CDMA_ERR_TIMEOUT = 7,            /* a bounded device-side wait ran out              */
+    CDMA_ERR_CUDA = 8,               /* a CUDA runtime call failed                      */
+    CDMA_ERR_OUT_OF_MEMORY = 9,      /* context pool exhausted / allocation failed      */
+    CDMA_ERR_BAD_TICKET = 10
+};
+
+/* element types: only the width matters to the codec (4, 2, 2 bytes) */
+enum { CDMA_F32 = 0, CDMA_F16 = 1, CDMA_BF16 = 2 };
+
+/* physical layouts of a 4-D activation map (Section II-C); a tag only */
+enum { CDMA_NCHW = 0, CDMA_NHWC = 1, CDMA_CHWN = 2 };
+
+#define CDMA_WINDOW 32u           /* elements per mask (Section V-A)              */
+#define CDMA_CHUNK 1024u          /* elements per offset-table entry              */
+
+const char* cdma_status_string(int status);
+
+/* Element width in bytes for a dtype code, 0 for an unknown code. */
+uint32_t cdma_dtype_size(int dtype);
+
+/* Worst-case payload size, 4*ceil(n/32) + s*n (every element non-zero: the
+ * all-ones mask plus 32 values per window, Section V-A), rounded up to a
+ * multiple of 16.  0 for an unknown dtype. */
+uint64_t cdma_zvc_max_compressed_bytes(uint64_t n, int dtype);
+
+/* Number of uint64 entries of the offset table: ceil(n/1024) + 1. */
+uint64_t cdma_zvc_table_entries(uint64_t n);
+
+/* Bytes of device scratch a codec call on n elements needs (both directions;
+ * a multiple of 256).  Holds the inter-tile prefix descriptors, the tile
+ * ticket and the status/result words. */
+uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype);
+
+/*
+ * Compress n elements at d_src into d_dst (payload) and d_table (offsets).
+ * One pass over the input: per window mask, per-window record sizes, running
+ * prefix across tiles, compaction (Section V-A; the engine's compare /
+ * prefix-sum / shift / append stages of Section V-B).
+ *
+ *   d_src           dense tensor, n*s bytes, 16-byte aligned, read only
+ *   dtype, layout   CDMA_F32/F16/BF16; CDMA_NCHW/NHWC/CHWN (tag)
+ *   d_dst           payload out; dst_capacity bytes, 16-byte aligned.  Any
+ *                   capacity is accepted; if the payload does not fit the
+ *                   call fails with BUFFER_TOO_SMALL having written only
+ *                   bytes below dst_capacity.
+ *   d_table         cdma_zvc_table_entries(n) uint64, 8-byte aligned
+ *   d_workspace     >= cdma_zvc_workspace_bytes(n, dtype), 16-byte aligned;
+ *                   contents on entry are irrelevant
+ *   cuda_stream     stream the work is enqueued on
+ *
+ * cdma_zvc_compress waits for the stream and returns the payload size C
+ * (Section V-D: the size is returned on completion).  n = 0 gives C = 0 and
+ * table = {0}.
+ *
+ * cdma_zvc_compress_async only enqueues.  h_result must point to two uint64
+ * in pinned host memory; once the stream reaches that point h_result[0] holds
+ * C and h_result[1] the status code (0 on success).
+ */
+int64_t cdma_zvc_compress(const void* d_src, uint64_t n, int dtype, int layout,
+                          void* d_dst, uint64_t dst_capacity, uint64_t* d_table,
+                          void* d_workspace, uint64_t workspace_bytes,
+                          void* cuda_stream);
+
+int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout,
+                            void* d_dst, uint64_t dst_capacity, uint64_t* d_table,
+                            void* d_workspace, uint64_t workspace_bytes,
+                            void* cuda_stream, uint64_t* h_result);
+
+/*
+ * Expand a payload back into n dense elements (Section V-B, decompression
+ * engine: the pop-count of a mask tells how many values its window takes,
+ * values or zeros are steered into place).
+ *
+ *   d_src, src_bytes   payload and its exact size C, 16-byte aligned
+ *   d_table            the offset table produced by compression
+ *   d_dst              n*s bytes out, 16-byte aligned
+ *   d_workspace        >= cdma_zvc_workspace_bytes(n, dtype)
+ *
+ * The table and every record are validated: offsets must be non-decreasing,
+ * inside the payload and a chunk must decode to exactly its byte range; a
+ * mask must not name an element at index >= n.  A violation gives
+ * CORRUPT_STREAM; no read leaves [d_src, d_src+src_bytes) and no write leaves
+ * the n elements regardless.
+ *
+ * cdma_zvc_decompress waits for the stream and returns n*s.
+ * cdma_zvc_decompress_async only enqueues; h_result as above, with
+ * h_result[0] = n*s.
+ */
+int64_t cdma_zvc_decompress(const void* d_src, uint64_t src_bytes,
+                            const uint64_t* d_table, uint64_t n, int dtype,
+                            int layout, void* d_dst, void* d_workspace,
+                            uint64_t workspace_bytes, void* cuda_stream);
+
+int cdma_zvc_decompress_async(const void* d_src, uint64_t src_bytes,
+                              const uint64_t* d_table, uint64_t n, int dtype,
+                              int layout, void* d_dst, void* d_workspace,
+                              uint64_t workspace_bytes, void* cuda_stream,
+                              uint64_t* h_result);
+
+/* ------------------------------------------------------------------------ *
+ * Offload pipeline (Section III, Fig. 2b: OFF(n) in the forward pass, PRE(n)
+ * in reverse order in the backward pass; Section V-D: the compressed copy
+ * replaces the cudaMemcpy calls of the memory manager).
+ * ------------------------------------------------------------------------ */
+typedef struct cdma_ctx cdma_ctx;
+typedef struct { uint64_t id; } cdma_ticket;
+
+/*
+ * Create a context on the current device.
+ *   pinned_bytes          size of the pinned host pool that holds offloaded
+ *                         payloads and their tables
+ *   device_staging_bytes  device memory for compressed staging; split into two
+ *                         slots so that one tensor's copy overlaps the next
+ *                         tensor's codec kernel.  A slot must hold the
+ *                         tensor's payload, table and workspace; sizing a slot
+ *                         for cdma_zvc_max_compressed_bytes of the largest
+ *                         tensor never fails, a smaller one fails with
+ *                         BUFFER_TOO_SMALL when a payload does not fit.
+ * All allocation happens here (and, for the host-buffer calls below, on the
+ * first call that needs a larger dense staging buffer).
+ */
+int cdma_ctx_create(uint64_t pinned_bytes, uint64_t device_staging_bytes, cdma_ctx** out);
+int cdma_ctx_destroy(cdma_ctx* ctx);
+
+/*
+ * OFF: compress the tensor on compute_stream into a staging slot, wait for
+ * the kernel (not for the copy), then enqueue the device-to-host copy of
+ * exactly C payload bytes plus the table on the context's side stream, into
+ * the pinned pool.  Returns C.  The copy proceeds while the caller continues;
+ * the next cdma_offload's kernel overlaps it.  d_src may be reused as soon as
+ * the call returns.
+ */
+int64_t cdma_offload(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, int layout,
+                     void* compute_stream, cdma_ticket* out);
+
+/*
+ * PRE: enqueue the host-to-device copy of the ticket's payload and table on
+ * the side stream, then the decompression into d_dst on compute_stream once
+ * the copy has landed.  The ticket and its pinned bytes are released.
+ * cdma_prefetch waits for the decompression and returns n*s (or -status);
+ * cdma_prefetch_async returns at once so the next tensor's copy overlaps this
+ * tensor's kernel; its outcome is reported by cdma_ctx_synchronize.
+ */
+int64_t cdma_prefetch(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream);
+int cdma_prefetch_async(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream);
+
+/* Wait for everything the context enqueued; returns the first deferred
+ * failure of an asynchronous call since the last synchronize, else 0. */
+int cdma_ctx_synchronize(cdma_ctx* ctx);
+
+/* Size facts of a live ticket: payload bytes and element count. 0 on success. */
+int cdma_ticket_info(cdma_ctx* ctx, cdma_ticket ticket, uint64_t* payload_bytes, uint64_t* n);
+
+/*
+ * The same compressed copies for callers whose tensors live in HOST memory
+ * (pinned for full speed): h_src is copied to the device, compressed, and the
+ * payload and table copied back into h_dst / h_table; and the reverse.  They
+ * run on the context's side stream, wait for completion and return C / n*s.
+ * h_table holds cdma_zvc_table_entries(n) uint64.
+ */
+int64_t cdma_zvc_compress_host(cdma_ctx* ctx, const void* h_src, uint64_t n, int dtype,
+                               int layout, void* h_dst, uint64_t dst_capacity,
+                               uint64_t* h_table);
+int64_t cdma_zvc_decompress_host(cdma_ctx* ctx, const void* h_src, uint64_t src_bytes,
+                                 const uint64_t* h_table, uint64_t n, int dtype, int layout,
+                                 void* h_dst);
+
+/* Number of kernel launches this library has issued in this process (codec
+ * kernels only; memsets and copies are not counted). */
+uint64_t cdma_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CDMA_H_ */
