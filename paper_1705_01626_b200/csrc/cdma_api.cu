@@ -1,0 +1,162 @@
+// extern "C" codec entry points: argument checking, workspace reset, launch,
+// result read-back.  Declarations and contracts are in include/cdma.h.
+#include <atomic>
+#include <cstring>
+
+#include "zvc_common.cuh"
+
+namespace cdma {
+
+static std::atomic<uint64_t> g_kernel_launches{0};
+void count_kernel_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
+
+static inline bool aligned(const void* p, uintptr_t a) {
+    return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0;
+}
+static inline bool overlaps(const void* a, uint64_t na, const void* b, uint64_t nb) {
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return na != 0 && nb != 0 && a0 < b0 + nb && b0 < a0 + na;
+}
+
+static int check_common(uint64_t n, int dtype, int layout, const void* dense, const void* packed,
+                        const uint64_t* table, const void* ws, uint64_t ws_bytes) {
+    const uint32_t s = cdma_dtype_size(dtype);
+    if (s == 0) return CDMA_ERR_UNSUPPORTED_DTYPE;
+    if (layout != CDMA_NCHW && layout != CDMA_NHWC && layout != CDMA_CHWN)
+        return CDMA_ERR_UNSUPPORTED_LAYOUT;
+    if (n > (1ull << 40)) return CDMA_ERR_INVALID_ARG;
+    if (table == nullptr || ws == nullptr) return CDMA_ERR_INVALID_ARG;
+    if (n != 0 && dense == nullptr) return CDMA_ERR_INVALID_ARG;
+    if (!aligned(dense, 16) || !aligned(packed, 16) || !aligned(ws, 16) || !aligned(table, 8))
+        return CDMA_ERR_ALIGNMENT;
+    if (ws_bytes < cdma_zvc_workspace_bytes(n, dtype)) return CDMA_ERR_BUFFER_TOO_SMALL;
+    return CDMA_OK;
+}
+
+}  // namespace cdma
+
+using namespace cdma;
+
+extern "C" {
+
+const char* cdma_status_string(int status) {
+    switch (status < 0 ? -status : status) {
+        case CDMA_OK: return "ok";
+        case CDMA_ERR_INVALID_ARG: return "invalid argument";
+        case CDMA_ERR_UNSUPPORTED_DTYPE: return "unsupported dtype";
+        case CDMA_ERR_UNSUPPORTED_LAYOUT: return "unsupported layout";
+        case CDMA_ERR_ALIGNMENT: return "buffer not 16-byte aligned";
+        case CDMA_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case CDMA_ERR_CORRUPT_STREAM: return "corrupt stream or offset table";
+        case CDMA_ERR_TIMEOUT: return "device-side wait ran out";
+        case CDMA_ERR_CUDA: return "CUDA runtime error";
+        case CDMA_ERR_OUT_OF_MEMORY: return "out of memory";
+        case CDMA_ERR_BAD_TICKET: return "unknown or consumed ticket";
+        default: return "unknown status";
+    }
+}
+
+uint32_t cdma_dtype_size(int dtype) {
+    switch (dtype) {
+        case CDMA_F32: return 4;
+        case CDMA_F16: return 2;
+        case CDMA_BF16: return 2;
+        default: return 0;
+    }
+}
+
+uint64_t cdma_zvc_max_compressed_bytes(uint64_t n, int dtype) {
+    const uint64_t s = cdma_dtype_size(dtype);
+    if (s == 0) return 0;
+    const uint64_t bytes = 4 * ((n + kWindow - 1) / kWindow) + s * n;
+    return (bytes + 15) & ~15ull;
+}
+
+uint64_t cdma_zvc_table_entries(uint64_t n) { return num_chunks_of(n) + 1; }
+
+uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype) {
+    (void)dtype;
+    const uint64_t bytes = kWsHeaderBytes + 8 * num_tiles_of(n);
+    return (bytes + 255) & ~255ull;
+}
+
+int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,
+                            uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
+                            uint64_t workspace_bytes, void* cuda_stream, uint64_t* h_result) {
+    const int st = check_common(n, dtype, layout, d_src, d_dst, d_table, d_workspace, workspace_bytes);
+    if (st != CDMA_OK) return st;
+    if (dst_capacity != 0 && d_dst == nullptr) return CDMA_ERR_INVALID_ARG;
+    if (h_result == nullptr) return CDMA_ERR_INVALID_ARG;
+    const uint32_t s = cdma_dtype_size(dtype);
+    if (overlaps(d_src, n * s, d_dst, dst_capacity)) return CDMA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint64_t* ws = static_cast<uint64_t*>(d_workspace);
+
+    // ticket, result words and every tile descriptor start at zero
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * num_tiles_of(n), stream) != cudaSuccess)
+        return CDMA_ERR_CUDA;
+    if (n == 0) {
+        if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    } else if (launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, stream) !=
+               cudaSuccess) {
+        return CDMA_ERR_CUDA;
+    }
+    if (cudaMemcpyAsync(h_result, ws + kWsBytes, 16, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return CDMA_ERR_CUDA;
+    return CDMA_OK;
+}
+
+int64_t cdma_zvc_compress(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,
+                          uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
+                          uint64_t workspace_bytes, void* cuda_stream) {
+    uint64_t result[2] = {0, 0};
+    const int st = cdma_zvc_compress_async(d_src, n, dtype, layout, d_dst, dst_capacity, d_table,
+                                           d_workspace, workspace_bytes, cuda_stream, result);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (result[1] != 0) return -static_cast<int64_t>(result[1]);
+    return static_cast<int64_t>(result[0]);
+}
+
+int cdma_zvc_decompress_async(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
+                              uint64_t n, int dtype, int layout, void* d_dst, void* d_workspace,
+                              uint64_t workspace_bytes, void* cuda_stream, uint64_t* h_result) {
+    const int st = check_common(n, dtype, layout, d_dst, d_src, d_table, d_workspace, workspace_bytes);
+    if (st != CDMA_OK) return st;
+    if (src_bytes != 0 && d_src == nullptr) return CDMA_ERR_INVALID_ARG;
+    if (h_result == nullptr) return CDMA_ERR_INVALID_ARG;
+    const uint32_t s = cdma_dtype_size(dtype);
+    if (overlaps(d_dst, n * s, d_src, src_bytes)) return CDMA_ERR_INVALID_ARG;
+    // sizes the format cannot produce are refused before anything is launched
+    const uint64_t windows = (n + kWindow - 1) / kWindow;
+    if (src_bytes < 4 * windows || src_bytes > 4 * windows + static_cast<uint64_t>(s) * n ||
+        src_bytes % s != 0)
+        return CDMA_ERR_CORRUPT_STREAM;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint64_t* ws = static_cast<uint64_t*>(d_workspace);
+
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    if (launch_zvc_decompress(d_src, src_bytes, d_table, n, s, d_dst, ws, stream) != cudaSuccess)
+        return CDMA_ERR_CUDA;
+    if (cudaMemcpyAsync(h_result, ws + kWsBytes, 16, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return CDMA_ERR_CUDA;
+    return CDMA_OK;
+}
+
+int64_t cdma_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
+                            uint64_t n, int dtype, int layout, void* d_dst, void* d_workspace,
+                            uint64_t workspace_bytes, void* cuda_stream) {
+    uint64_t result[2] = {0, 0};
+    const int st = cdma_zvc_decompress_async(d_src, src_bytes, d_table, n, dtype, layout, d_dst,
+                                             d_workspace, workspace_bytes, cuda_stream, result);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (result[1] != 0) return -static_cast<int64_t>(result[1]);
+    return static_cast<int64_t>(n) * cdma_dtype_size(dtype);
+}
+
+uint64_t cdma_kernel_launch_count(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,425 @@
+// Offload / prefetch pipeline (Section III, Fig. 2b; Section V-D): OFF(n)
+// compresses an activation map and copies the compressed bytes to pinned host
+// memory, PRE(n) copies them back and expands them.  The codec kernels run on
+// the caller's compute stream, the copies on a side stream owned by the
+// context; two device staging slots let one tensor's copy overlap the next
+// tensor's kernel.  Host code only: contracts are in include/cdma.h.
+#include <map>
+#include <new>
+#include <unordered_map>
+#include <vector>
+
+#include "zvc_common.cuh"
+
+namespace {
+
+constexpr uint64_t kAlign = 256;
+constexpr uint32_t kSlots = 2;
+constexpr uint32_t kResultRing = 1024;   // pinned {bytes,status} pairs for asynchronous calls
+
+inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+// First-fit allocator over the pinned pool with merging of free neighbours.
+class RegionPool {
+public:
+    void reset(uint64_t bytes) {
+        free_.clear();
+        if (bytes) free_[0] = bytes;
+    }
+    bool alloc(uint64_t bytes, uint64_t* off) {
+        bytes = round_up(bytes ? bytes : 1, kAlign);
+        for (auto it = free_.begin(); it != free_.end(); ++it) {
+            if (it->second >= bytes) {
+                *off = it->first;
+                const uint64_t rest = it->second - bytes;
+                const uint64_t rest_off = it->first + bytes;
+                free_.erase(it);
+                if (rest) free_[rest_off] = rest;
+                return true;
+            }
+        }
+        return false;
+    }
+    void release(uint64_t off, uint64_t bytes) {
+        bytes = round_up(bytes ? bytes : 1, kAlign);
+        auto it = free_.emplace(off, bytes).first;
+        auto next = std::next(it);
+        if (next != free_.end() && it->first + it->second == next->first) {
+            it->second += next->second;
+            free_.erase(next);
+        }
+        if (it != free_.begin()) {
+            auto prev = std::prev(it);
+            if (prev->first + prev->second == it->first) {
+                prev->second += it->second;
+                free_.erase(it);
+            }
+        }
+    }
+
+private:
+    std::map<uint64_t, uint64_t> free_;
+};
+
+struct Slot {
+    uint8_t* base = nullptr;
+    uint64_t bytes = 0;
+    cudaEvent_t idle = nullptr;     // last use of the slot has finished
+    cudaEvent_t staged = nullptr;   // kernel (offload) / copy (prefetch) into the slot has finished
+    bool used = false;
+};
+
+struct SlotPlan {
+    uint64_t* table;
+    uint64_t table_bytes;
+    uint64_t* ws;
+    uint64_t ws_bytes;
+    uint8_t* payload;
+    uint64_t capacity;
+};
+
+struct TicketRec {
+    uint64_t n;
+    int dtype, layout;
+    uint64_t payload_bytes;
+    uint64_t pool_off, pool_bytes;
+};
+
+}  // namespace
+
+struct cdma_ctx {
+    int device = 0;
+    cudaStream_t side = nullptr;
+    uint8_t* h_pool = nullptr;
+    uint64_t pool_bytes = 0;
+    RegionPool pool;
+    uint8_t* d_staging = nullptr;
+    Slot slots[kSlots];
+    uint32_t next_slot = 0;
+    std::unordered_map<uint64_t, TicketRec> tickets;
+    uint64_t next_ticket = 1;
+    uint64_t* h_results = nullptr;
+    uint32_t next_result = 0;
+    std::vector<uint64_t*> pending;   // results of asynchronous calls not yet inspected
+    int deferred = 0;
+    void* d_dense = nullptr;          // dense staging of the host-buffer calls
+    uint64_t dense_bytes = 0;
+};
+
+namespace {
+
+bool plan_slot(const Slot& slot, uint64_t n, int dtype, SlotPlan* p) {
+    p->table_bytes = 8 * cdma_zvc_table_entries(n);
+    p->ws_bytes = cdma_zvc_workspace_bytes(n, dtype);
+    const uint64_t head = round_up(p->table_bytes, kAlign) + round_up(p->ws_bytes, kAlign);
+    if (slot.bytes < head) return false;
+    p->table = reinterpret_cast<uint64_t*>(slot.base);
+    p->ws = reinterpret_cast<uint64_t*>(slot.base + round_up(p->table_bytes, kAlign));
+    p->payload = slot.base + head;
+    const uint64_t room = (slot.bytes - head) & ~15ull;
+    const uint64_t worst = cdma_zvc_max_compressed_bytes(n, dtype);
+    p->capacity = room < worst ? room : worst;
+    return true;
+}
+
+uint64_t* next_result_words(cdma_ctx* ctx) {
+    uint64_t* r = ctx->h_results + 2 * (ctx->next_result % kResultRing);
+    ++ctx->next_result;
+    r[0] = 0;
+    r[1] = 0;
+    return r;
+}
+
+// Inspect finished asynchronous calls; keeps the first failure.
+void collect_pending(cdma_ctx* ctx) {
+    for (uint64_t* r : ctx->pending)
+        if (r[1] != 0 && ctx->deferred == 0) ctx->deferred = static_cast<int>(r[1]);
+    ctx->pending.clear();
+}
+
+int wait_all(cdma_ctx* ctx) {
+    if (cudaStreamSynchronize(ctx->side) != cudaSuccess) return CDMA_ERR_CUDA;
+    for (Slot& s : ctx->slots)
+        if (s.used && cudaEventSynchronize(s.idle) != cudaSuccess) return CDMA_ERR_CUDA;
+    collect_pending(ctx);
+    return CDMA_OK;
+}
+
+int ensure_dense(cdma_ctx* ctx, uint64_t bytes) {
+    if (bytes <= ctx->dense_bytes) return CDMA_OK;
+    if (wait_all(ctx) != CDMA_OK) return CDMA_ERR_CUDA;
+    if (ctx->d_dense) cudaFree(ctx->d_dense);
+    ctx->d_dense = nullptr;
+    ctx->dense_bytes = 0;
+    if (cudaMalloc(&ctx->d_dense, round_up(bytes, kAlign)) != cudaSuccess) {
+        cudaGetLastError();
+        return CDMA_ERR_OUT_OF_MEMORY;
+    }
+    ctx->dense_bytes = round_up(bytes, kAlign);
+    return CDMA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int cdma_ctx_create(uint64_t pinned_bytes, uint64_t device_staging_bytes, cdma_ctx** out) {
+    if (out == nullptr) return CDMA_ERR_INVALID_ARG;
+    *out = nullptr;
+    cdma_ctx* ctx = new (std::nothrow) cdma_ctx();
+    if (ctx == nullptr) return CDMA_ERR_OUT_OF_MEMORY;
+    int st = CDMA_OK;
+    const uint64_t slot_bytes = (device_staging_bytes / kSlots) & ~(kAlign - 1);
+    do {
+        if (cudaGetDevice(&ctx->device) != cudaSuccess) { st = CDMA_ERR_CUDA; break; }
+        if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess) {
+            st = CDMA_ERR_CUDA; break;
+        }
+        if (pinned_bytes &&
+            cudaHostAlloc(reinterpret_cast<void**>(&ctx->h_pool), pinned_bytes, cudaHostAllocDefault) !=
+                cudaSuccess) {
+            st = CDMA_ERR_OUT_OF_MEMORY; break;
+        }
+        ctx->pool_bytes = pinned_bytes;
+        ctx->pool.reset(pinned_bytes);
+        if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->h_results), 16 * kResultRing,
+                          cudaHostAllocDefault) != cudaSuccess) {
+            st = CDMA_ERR_OUT_OF_MEMORY; break;
+        }
+        if (slot_bytes &&
+            cudaMalloc(reinterpret_cast<void**>(&ctx->d_staging), slot_bytes * kSlots) != cudaSuccess) {
+            st = CDMA_ERR_OUT_OF_MEMORY; break;
+        }
+        for (uint32_t i = 0; i < kSlots && st == CDMA_OK; ++i) {
+            ctx->slots[i].base = ctx->d_staging ? ctx->d_staging + i * slot_bytes : nullptr;
+            ctx->slots[i].bytes = slot_bytes;
+            if (cudaEventCreateWithFlags(&ctx->slots[i].idle, cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&ctx->slots[i].staged, cudaEventDisableTiming) != cudaSuccess)
+                st = CDMA_ERR_CUDA;
+        }
+    } while (false);
+    if (st != CDMA_OK) {
+        cudaGetLastError();
+        cdma_ctx_destroy(ctx);
+        return st;
+    }
+    *out = ctx;
+    return CDMA_OK;
+}
+
+int cdma_ctx_destroy(cdma_ctx* ctx) {
+    if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
+    if (ctx->side) cudaStreamSynchronize(ctx->side);
+    for (Slot& s : ctx->slots) {
+        if (s.used && s.idle) cudaEventSynchronize(s.idle);
+        if (s.idle) cudaEventDestroy(s.idle);
+        if (s.staged) cudaEventDestroy(s.staged);
+    }
+    if (ctx->d_dense) cudaFree(ctx->d_dense);
+    if (ctx->d_staging) cudaFree(ctx->d_staging);
+    if (ctx->h_results) cudaFreeHost(ctx->h_results);
+    if (ctx->h_pool) cudaFreeHost(ctx->h_pool);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
+    delete ctx;
+    return CDMA_OK;
+}
+
+int64_t cdma_offload(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, int layout,
+                     void* compute_stream, cdma_ticket* out) {
+    if (ctx == nullptr || out == nullptr) return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
+    if (cdma_dtype_size(dtype) == 0) return -static_cast<int64_t>(CDMA_ERR_UNSUPPORTED_DTYPE);
+    cudaStream_t compute = static_cast<cudaStream_t>(compute_stream);
+    Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
+    SlotPlan p;
+    if (!plan_slot(slot, n, dtype, &p)) return -static_cast<int64_t>(CDMA_ERR_BUFFER_TOO_SMALL);
+
+    // the slot's previous copy must have drained before the kernel overwrites it
+    if (slot.used && cudaStreamWaitEvent(compute, slot.idle, 0) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    uint64_t* res = next_result_words(ctx);
+    const int st = cdma_zvc_compress_async(d_src, n, dtype, layout, p.payload, p.capacity, p.table, p.ws,
+                                           p.ws_bytes, compute, res);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (cudaEventRecord(slot.staged, compute) != cudaSuccess ||
+        cudaEventSynchronize(slot.staged) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    slot.used = true;
+    cudaEventRecord(slot.idle, compute);
+    if (res[1] != 0) return -static_cast<int64_t>(res[1]);
+    const uint64_t c = res[0];
+
+    // exactly C payload bytes and the table cross the link (Section V-D: the
+    // compressed size is known on completion and sizes the host allocation)
+    TicketRec rec{n, dtype, layout, c, 0, round_up(c, 16) + p.table_bytes};
+    if (!ctx->pool.alloc(rec.pool_bytes, &rec.pool_off) ||
+        rec.pool_off + rec.pool_bytes > ctx->pool_bytes)
+        return -static_cast<int64_t>(CDMA_ERR_OUT_OF_MEMORY);
+    uint8_t* h = ctx->h_pool + rec.pool_off;
+    bool ok = true;
+    if (c) ok &= cudaMemcpyAsync(h, p.payload, c, cudaMemcpyDeviceToHost, ctx->side) == cudaSuccess;
+    ok &= cudaMemcpyAsync(h + round_up(c, 16), p.table, p.table_bytes, cudaMemcpyDeviceToHost,
+                          ctx->side) == cudaSuccess;
+    ok &= cudaEventRecord(slot.idle, ctx->side) == cudaSuccess;
+    if (!ok) {
+        ctx->pool.release(rec.pool_off, rec.pool_bytes);
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    }
+    out->id = ctx->next_ticket++;
+    ctx->tickets[out->id] = rec;
+    return static_cast<int64_t>(c);
+}
+
+static int prefetch_enqueue(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream,
+                            Slot** used_slot, uint64_t** result, uint64_t* dense_bytes) {
+    if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
+    auto it = ctx->tickets.find(ticket.id);
+    if (it == ctx->tickets.end()) return CDMA_ERR_BAD_TICKET;
+    const TicketRec rec = it->second;
+    cudaStream_t compute = static_cast<cudaStream_t>(compute_stream);
+    if (ctx->pending.size() + 2 >= kResultRing) {
+        if (wait_all(ctx) != CDMA_OK) return CDMA_ERR_CUDA;
+    }
+    Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
+    SlotPlan p;
+    if (!plan_slot(slot, rec.n, rec.dtype, &p) || p.capacity < rec.payload_bytes)
+        return CDMA_ERR_BUFFER_TOO_SMALL;
+    if (slot.used && cudaStreamWaitEvent(ctx->side, slot.idle, 0) != cudaSuccess) return CDMA_ERR_CUDA;
+    const uint8_t* h = ctx->h_pool + rec.pool_off;
+    bool ok = true;
+    if (rec.payload_bytes)
+        ok &= cudaMemcpyAsync(p.payload, h, rec.payload_bytes, cudaMemcpyHostToDevice, ctx->side) ==
+              cudaSuccess;
+    ok &= cudaMemcpyAsync(p.table, h + round_up(rec.payload_bytes, 16), p.table_bytes,
+                          cudaMemcpyHostToDevice, ctx->side) == cudaSuccess;
+    ok &= cudaEventRecord(slot.staged, ctx->side) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(compute, slot.staged, 0) == cudaSuccess;
+    if (!ok) return CDMA_ERR_CUDA;
+    slot.used = true;
+    cudaEventRecord(slot.idle, ctx->side);
+    uint64_t* res = next_result_words(ctx);
+    const int st = cdma_zvc_decompress_async(p.payload, rec.payload_bytes, p.table, rec.n, rec.dtype,
+                                             rec.layout, d_dst, p.ws, p.ws_bytes, compute, res);
+    if (st != CDMA_OK) return st;   // the ticket stays valid: nothing was consumed
+    if (cudaEventRecord(slot.idle, compute) != cudaSuccess) return CDMA_ERR_CUDA;
+    // Later copies into this pinned region are enqueued on the same side
+    // stream, behind the copy just issued, so the region can be recycled now.
+    ctx->pool.release(rec.pool_off, rec.pool_bytes);
+    ctx->tickets.erase(it);
+    *used_slot = &slot;
+    *result = res;
+    *dense_bytes = rec.n * cdma_dtype_size(rec.dtype);
+    return CDMA_OK;
+}
+
+int cdma_prefetch_async(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream) {
+    Slot* slot = nullptr;
+    uint64_t* res = nullptr;
+    uint64_t dense = 0;
+    const int st = prefetch_enqueue(ctx, ticket, d_dst, compute_stream, &slot, &res, &dense);
+    if (st == CDMA_OK) ctx->pending.push_back(res);
+    return st;
+}
+
+int64_t cdma_prefetch(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream) {
+    Slot* slot = nullptr;
+    uint64_t* res = nullptr;
+    uint64_t dense = 0;
+    const int st = prefetch_enqueue(ctx, ticket, d_dst, compute_stream, &slot, &res, &dense);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (cudaEventSynchronize(slot->idle) != cudaSuccess) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (res[1] != 0) return -static_cast<int64_t>(res[1]);
+    return static_cast<int64_t>(dense);
+}
+
+int cdma_ctx_synchronize(cdma_ctx* ctx) {
+    if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
+    const int st = wait_all(ctx);
+    if (st != CDMA_OK) return st;
+    const int d = ctx->deferred;
+    ctx->deferred = 0;
+    return d;
+}
+
+int cdma_ticket_info(cdma_ctx* ctx, cdma_ticket ticket, uint64_t* payload_bytes, uint64_t* n) {
+    if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
+    auto it = ctx->tickets.find(ticket.id);
+    if (it == ctx->tickets.end()) return CDMA_ERR_BAD_TICKET;
+    if (payload_bytes) *payload_bytes = it->second.payload_bytes;
+    if (n) *n = it->second.n;
+    return CDMA_OK;
+}
+
+int64_t cdma_zvc_compress_host(cdma_ctx* ctx, const void* h_src, uint64_t n, int dtype, int layout,
+                               void* h_dst, uint64_t dst_capacity, uint64_t* h_table) {
+    if (ctx == nullptr || h_table == nullptr || (n && h_src == nullptr) ||
+        (dst_capacity && h_dst == nullptr))
+        return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
+    const uint32_t s = cdma_dtype_size(dtype);
+    if (s == 0) return -static_cast<int64_t>(CDMA_ERR_UNSUPPORTED_DTYPE);
+    int st = ensure_dense(ctx, n * s);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
+    SlotPlan p;
+    if (!plan_slot(slot, n, dtype, &p)) return -static_cast<int64_t>(CDMA_ERR_BUFFER_TOO_SMALL);
+    if (slot.used && cudaStreamWaitEvent(ctx->side, slot.idle, 0) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (n && cudaMemcpyAsync(ctx->d_dense, h_src, n * s, cudaMemcpyHostToDevice, ctx->side) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    uint64_t* res = next_result_words(ctx);
+    st = cdma_zvc_compress_async(ctx->d_dense, n, dtype, layout, p.payload, p.capacity, p.table, p.ws,
+                                 p.ws_bytes, ctx->side, res);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    slot.used = true;
+    cudaEventRecord(slot.idle, ctx->side);
+    if (cudaStreamSynchronize(ctx->side) != cudaSuccess) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (res[1] != 0) return -static_cast<int64_t>(res[1]);
+    const uint64_t c = res[0];
+    if (c > dst_capacity) return -static_cast<int64_t>(CDMA_ERR_BUFFER_TOO_SMALL);
+    bool ok = true;
+    if (c) ok &= cudaMemcpyAsync(h_dst, p.payload, c, cudaMemcpyDeviceToHost, ctx->side) == cudaSuccess;
+    ok &= cudaMemcpyAsync(h_table, p.table, p.table_bytes, cudaMemcpyDeviceToHost, ctx->side) ==
+          cudaSuccess;
+    ok &= cudaEventRecord(slot.idle, ctx->side) == cudaSuccess;
+    ok &= cudaStreamSynchronize(ctx->side) == cudaSuccess;
+    if (!ok) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    return static_cast<int64_t>(c);
+}
+
+int64_t cdma_zvc_decompress_host(cdma_ctx* ctx, const void* h_src, uint64_t src_bytes,
+                                 const uint64_t* h_table, uint64_t n, int dtype, int layout,
+                                 void* h_dst) {
+    if (ctx == nullptr || h_table == nullptr || (src_bytes && h_src == nullptr) ||
+        (n && h_dst == nullptr))
+        return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
+    const uint32_t s = cdma_dtype_size(dtype);
+    if (s == 0) return -static_cast<int64_t>(CDMA_ERR_UNSUPPORTED_DTYPE);
+    int st = ensure_dense(ctx, n * s);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
+    SlotPlan p;
+    if (!plan_slot(slot, n, dtype, &p) || p.capacity < src_bytes)
+        return -static_cast<int64_t>(src_bytes > cdma_zvc_max_compressed_bytes(n, dtype)
+                                         ? CDMA_ERR_CORRUPT_STREAM
+                                         : CDMA_ERR_BUFFER_TOO_SMALL);
+    if (slot.used && cudaStreamWaitEvent(ctx->side, slot.idle, 0) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    bool ok = true;
+    if (src_bytes)
+        ok &= cudaMemcpyAsync(p.payload, h_src, src_bytes, cudaMemcpyHostToDevice, ctx->side) == cudaSuccess;
+    ok &= cudaMemcpyAsync(p.table, h_table, p.table_bytes, cudaMemcpyHostToDevice, ctx->side) == cudaSuccess;
+    if (!ok) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    uint64_t* res = next_result_words(ctx);
+    st = cdma_zvc_decompress_async(p.payload, src_bytes, p.table, n, dtype, layout, ctx->d_dense, p.ws,
+                                   p.ws_bytes, ctx->side, res);
+    slot.used = true;
+    cudaEventRecord(slot.idle, ctx->side);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (n) ok &= cudaMemcpyAsync(h_dst, ctx->d_dense, n * s, cudaMemcpyDeviceToHost, ctx->side) == cudaSuccess;
+    ok &= cudaEventRecord(slot.idle, ctx->side) == cudaSuccess;
+    ok &= cudaStreamSynchronize(ctx->side) == cudaSuccess;
+    if (!ok) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (res[1] != 0) return -static_cast<int64_t>(res[1]);
+    return static_cast<int64_t>(n * s);
+}
+
+}  // extern "C"

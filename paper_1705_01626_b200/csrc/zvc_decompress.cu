@@ -1,0 +1,124 @@
+// Zero-value decompression (Section V-B, Fig. 10b): the pop-count of a mask
+// tells how many payload values its window takes; values or zeros are steered
+// into the window's 32 places.
+//
+// One warp expands one chunk (1024 elements).  The offset table gives the
+// chunk's byte range in the payload; the warp copies that range into shared
+// memory with 16-byte loads, then walks the records: the position of window
+// w+1's mask is the position of window w's mask plus 4 plus s times the
+// pop-count of that mask (the stream is self-delimiting, Section V-A).  Lane =
+// element: a lane whose mask bit is set reads the value at its rank among the
+// set bits below it, the others write zero; every window is one coalesced
+// store.  The table and every record are validated; nothing is read outside
+// the payload or written outside the tensor whatever the input holds.
+#include "zvc_common.cuh"
+
+namespace cdma {
+
+namespace {
+
+constexpr uint32_t kDecWarps = 8;
+constexpr uint32_t kDecThreads = 32 * kDecWarps;
+
+template <typename T>
+__global__ void __launch_bounds__(kDecThreads)
+zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
+                      const uint64_t* __restrict__ table, uint64_t n, T* __restrict__ dst,
+                      uint64_t* __restrict__ ws, uint64_t num_chunks) {
+    constexpr uint32_t S = sizeof(T);
+    constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
+    constexpr uint32_t kBuf = kMaxChunkBytes + 32;   // 16-byte phase in front, round-up behind
+    __shared__ __align__(16) uint8_t s_buf[kDecWarps][kBuf];
+
+    const uint32_t lane = lane_id();
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * kDecWarps + warp;
+    if (blockIdx.x == 0 && threadIdx.x == 0) ws[kWsBytes] = n * S;
+    if (chunk >= num_chunks) return;
+
+    const uint64_t e0 = chunk * kChunk;
+    const uint32_t nelem = (n - e0 < kChunk) ? static_cast<uint32_t>(n - e0) : kChunk;
+    const uint32_t nwin = (nelem + kWindow - 1) / kWindow;
+
+    // ---- the chunk's byte range, validated ----------------------------------
+    const uint64_t lo = __ldg(table + chunk);
+    const uint64_t hi = __ldg(table + chunk + 1);
+    bool ok = (lo <= hi) && (hi <= src_bytes) && (hi - lo >= 4ull * nwin) &&
+              (hi - lo <= 4ull * nwin + static_cast<uint64_t>(S) * nelem) && (lo % S == 0) &&
+              ((hi - lo) % S == 0);
+    if (chunk == 0 && lo != 0) ok = false;
+    if (chunk == num_chunks - 1 && hi != src_bytes) ok = false;
+    if (!ok) {
+        if (lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+        return;
+    }
+
+    // ---- stage payload bytes [lo, hi) in shared memory -----------------------
+    uint8_t* buf = s_buf[warp];
+    const uint64_t a0 = lo & ~15ull;              // buf[0] corresponds to payload byte a0
+    for (uint64_t a = a0 + 16ull * lane; a < hi; a += 16ull * 32) {
+        uint4 q;
+        if (a + 16 <= src_bytes) {
+            q = __ldcs(reinterpret_cast<const uint4*>(src + a));
+        } else {
+            // last, partial 16 bytes of the payload: never read past src_bytes
+            uint32_t wds[4] = {0, 0, 0, 0};
+            for (uint32_t b = 0; b < 16; b += 2) {
+                if (a + b + 2 <= src_bytes) {
+                    const uint32_t h = *reinterpret_cast<const uint16_t*>(src + a + b);
+                    wds[b >> 2] |= h << (8 * (b & 2));
+                }
+            }
+            q = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+        }
+        *reinterpret_cast<uint4*>(buf + (a - a0)) = q;
+    }
+    __syncwarp();
+
+    // ---- walk the records and expand ----------------------------------------
+    const T* units = reinterpret_cast<const T*>(buf);
+    uint32_t p = static_cast<uint32_t>(lo - a0) / S;        // position in units of S bytes
+    const uint32_t end = static_cast<uint32_t>(hi - a0) / S;
+    const uint32_t lt = lanemask_lt();
+    bool bad = false;
+    T* out = dst + e0 + lane;
+#pragma unroll 8
+    for (uint32_t w = 0; w < nwin; ++w) {
+        if (p + 4 / S > end) { bad = true; break; }
+        uint32_t m;
+        if (S == 4) m = units[p];
+        else m = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
+        const uint32_t cnt = __popc(m);
+        const uint32_t left = nelem - w * kWindow;           // elements this window really has
+        if (p + 4 / S + cnt > end || (left < kWindow && (m >> left) != 0)) { bad = true; break; }
+        const bool bit = (m >> lane) & 1u;
+        const T val = bit ? units[p + 4 / S + __popc(m & lt)] : T(0);
+        if (lane < left) __stcs(out + w * kWindow, val);
+        p += 4 / S + cnt;
+    }
+    if (!bad && p != end) bad = true;
+    if (bad && lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+}
+
+}  // namespace
+
+cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
+                                  uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
+                                  cudaStream_t stream) {
+    const uint64_t chunks = num_chunks_of(n);
+    if (chunks == 0) return cudaSuccess;
+    const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
+    if (elem_size == 4) {
+        zvc_decompress_kernel<uint32_t><<<grid, kDecThreads, 0, stream>>>(
+            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint32_t*>(d_dst),
+            d_ws, chunks);
+    } else {
+        zvc_decompress_kernel<uint16_t><<<grid, kDecThreads, 0, stream>>>(
+            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint16_t*>(d_dst),
+            d_ws, chunks);
+    }
+    count_kernel_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace cdma
