@@ -1,0 +1,551 @@
+#!/usr/bin/env python
+"""Benchmark of the ZVC codec hot path on B200: one JSON line on stdout.
+
+A step is one pass of the whole hot path over one activation map: compress
+(load, mask, scan, look-back, compaction, table) then decompress (table read,
+staging, mask walk, expansion).  The default workload is the VGG-16
+conv1_2-shaped fp32 map (64x64x224x224, 822 MB, per-channel Beta(2,4)
+densities); other workloads can be chosen with --workload for the results
+table.  Inputs are synthetic and seeded; they are larger than L2 so every step
+streams from HBM.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl cdma|reference]
+                  [--workload NAME]
+
+N > 1 is launched under torchrun, one rank per GPU.  The codec has no exchange
+step: every rank compresses its own tensor (weak scaling, no collective on the
+data path).
+
+--impl reference times the CPU oracle (the plain C checker) on the host cores,
+on bounded samples of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "zvc_compress_decompress_uncompressed_GBps"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+# DRAM bytes per launch measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum),
+# as a multiple of the algorithmic bytes of the same launch; see the summaries
+# under profiles/.  None until a capture exists for the kernel.
+NCU_TRAFFIC_FACTOR = {"zvc_compress_kernel": None, "zvc_decompress_kernel": None}
+
+
+def env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- #
+# workloads
+# --------------------------------------------------------------------------- #
+def make_workload(name: str, device, rank: int = 0):
+    """Returns (tensor, description).  Rank r > 0 draws a different seed."""
+    import torch
+    from paper_1705_01626_b200 import workloads as wl
+    bump = 7919 * rank
+    if name == "config1":
+        return wl.alexnet_conv1(seed=wl.seed_for(1) + bump, device=device), \
+            "config1: fp32 NCHW 32x96x55x55, i.i.d. density 0.5"
+    if name == "config2":
+        return wl.per_channel_beta(seed=wl.seed_for(2) + bump, device=device), \
+            "config2: fp32 NCHW 64x64x224x224 (VGG-16 conv1_2), per-channel Beta(2,4) density"
+    if name in ("config5a", "config5b", "config5c"):
+        which = name[-1]
+        x = wl.large_extremes(which, device=device, seed=wl.seed_for(5, "abc".index(which)) + bump)
+        return x, {"a": "config5a: fp32 2^29 elements, i.i.d. density 0.05",
+                   "b": "config5b: fp32 2^29 elements, all non-zero",
+                   "c": "config5c: fp16 2^29 elements, i.i.d. density 0.3"}[which]
+    if name.startswith("config3."):
+        i = int(name.split(".")[1])
+        c, h, w = wl.VGG16_CONV_SHAPES[i]
+        d = 0.5 - 0.4 * i / 12
+        return wl.correlated_relu((64, c, h, w), d, wl.seed_for(3, i) + bump, device), \
+            "config3 tensor %d: fp32 NCHW 64x%dx%dx%d, clustered zeros, density %.3f" % (i, c, h, w, d)
+    if name.startswith("iid:"):
+        # iid:<elements>:<density>[:f16] -- free-size case for profiling and sweeps
+        parts = name.split(":")
+        cnt, d = int(parts[1]), float(parts[2])
+        dt = torch.float16 if len(parts) > 3 and parts[3] == "f16" else torch.float32
+        return wl.iid_relu_like((cnt,), d, wl.seed_for(9) + bump, device, dtype=dt, floor=2.0 ** -10), \
+            "iid: %s %d elements, i.i.d. density %g" % ("fp16" if dt == torch.float16 else "fp32", cnt, d)
+    raise SystemExit("unknown workload %r" % name)
+
+
+# --------------------------------------------------------------------------- #
+# clock sampling during the timed region (read-only NVML queries)
+# --------------------------------------------------------------------------- #
+class ClockSampler:
+    REASONS = {
+        0x0000000000000004: "sw_power_cap",
+        0x0000000000000008: "hw_slowdown",
+        0x0000000000000020: "sw_thermal_slowdown",
+        0x0000000000000040: "hw_thermal_slowdown",
+        0x0000000000000080: "hw_power_brake_slowdown",
+    }
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.005)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+# --------------------------------------------------------------------------- #
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# --------------------------------------------------------------------------- #
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+class OracleRunner:
+    """Times the C oracle's compress and decompress on one sample with buffers
+    allocated (and touched) beforehand, so only the two C calls are timed."""
+
+    def __init__(self, sample, threads: int):
+        import numpy as np
+        from oracle import zvc_c
+        self.zvc_c, self.sample, self.threads = zvc_c, sample, threads
+        n, s = sample.size, sample.dtype.itemsize
+        self.dst = np.zeros(4 * ((n + 31) // 32) + s * n, dtype=np.uint8)
+        self.table = np.zeros(zvc_c.table_entries(n), dtype=np.uint64)
+        self.out = np.zeros(n, dtype=sample.dtype)
+        self.checked = False
+
+    def round_trip(self):
+        """Returns (compress seconds, decompress seconds, payload bytes)."""
+        t0 = time.perf_counter()
+        c = self.zvc_c.compress_into(self.sample, self.dst, self.table, self.threads)
+        t1 = time.perf_counter()
+        r = self.zvc_c.decompress_into(self.dst[:max(c, 0)], self.table, self.out, self.threads)
+        t2 = time.perf_counter()
+        if c < 0 or r != self.sample.nbytes:
+            raise SystemExit("oracle failed: %d %d" % (c, r))
+        if not self.checked:
+            assert self.out.tobytes() == self.sample.tobytes()
+            self.checked = True
+        return t1 - t0, t2 - t1, c
+
+
+def time_oracle_round_trip(sample, threads: int):
+    return OracleRunner(sample, threads).round_trip()
+
+
+def oracle_sample_elems(host_flat, threads: int, target_seconds: float) -> int:
+    """Pick a sample size (multiple of 1024 elements) costing about target_seconds."""
+    probe = min(host_flat.size, 4 << 20)
+    tc, td, _ = time_oracle_round_trip(host_flat[:probe], threads)
+    rate = probe / max(tc + td, 1e-9)
+    n = int(rate * target_seconds) // 1024 * 1024
+    return max(1024, min(n, host_flat.size // 1024 * 1024 or host_flat.size))
+
+
+def cpu_baseline(host_flat, target_seconds: float = 12.0):
+    """The C oracle on all host cores over a bounded sample, repeated until
+    about target_seconds of CPU wall time have been spent."""
+    threads = host_cores()
+    n = oracle_sample_elems(host_flat, threads, target_seconds)
+    sample = host_flat[:n]
+    runner = OracleRunner(sample, threads)
+    runner.round_trip()                      # untimed: touches every buffer once
+    tc = td = 0.0
+    reps = 0
+    while reps < 1 or (tc + td < target_seconds and reps < 200):
+        a, b, c = runner.round_trip()
+        tc, td, reps = tc + a, td + b, reps + 1
+    total = sample.nbytes * reps
+    one = OracleRunner(sample[: min(n, 8 << 20)], 1)
+    one.round_trip()
+    a1, b1, _ = one.round_trip()
+    return {
+        "value": total / (tc + td) / 1e9,
+        "unit": UNIT,
+        "cores": threads,
+        "kind": "oracle",
+        "sample": "first %d elements (%.1f MB) of the same tensor, %d round trips, compress %.2f s + "
+                  "decompress %.2f s in total, chunk-parallel driver over the byte-wise C oracle"
+                  % (n, sample.nbytes / 1e6, reps, tc, td),
+        "compress_GBps": total / tc / 1e9,
+        "decompress_GBps": total / td / 1e9,
+        "single_thread_GBps": one.sample.nbytes / (a1 + b1) / 1e9,
+    }
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle as it stands, on bounded samples."""
+    rank = env_int("RANK", 0)
+    if rank != 0:
+        return
+    import torch
+    x, desc = make_workload(args.workload, "cpu") if args.workload == "config1" else (None, None)
+    if x is None:
+        # generate a bounded slice of the workload's recipe on the CPU: the first
+        # images of the batch (same per-channel statistics), enough for the samples
+        from paper_1705_01626_b200 import workloads as wl
+        if args.workload == "config2":
+            x = wl.per_channel_beta(shape=(8, 64, 224, 224), device="cpu")
+            desc = "config2: fp32 NCHW 64x64x224x224 (VGG-16 conv1_2), per-channel Beta(2,4) density"
+        else:
+            x, desc = make_workload(args.workload, "cpu")
+    host = x.contiguous().view(-1).numpy()
+    threads = host_cores()
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    n = oracle_sample_elems(host, threads, min(budget, 15.0))
+    sample = host[:n]
+    runner = OracleRunner(sample, threads)
+    for _ in range(args.warmup):
+        runner.round_trip()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        runner.round_trip()
+    dt = time.perf_counter() - t0
+    value = sample.nbytes * args.steps / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
+        "data": "synthetic", "config": {"workload": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": "each step = first %d elements (%.1f MB) of the workload's recipe" %
+                                   (n, sample.nbytes / 1e6)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- #
+# the CUDA arm
+# --------------------------------------------------------------------------- #
+def run_cdma(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1705_01626_b200 import binding as B
+
+    world = env_int("WORLD_SIZE", 1)
+    rank = env_int("RANK", 0)
+    local = env_int("LOCAL_RANK", 0)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the codec has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    x, desc = make_workload(args.workload, dev, rank)
+    x = x.contiguous()
+    n, s = x.numel(), x.element_size()
+    code = {torch.float32: B.F32, torch.float16: B.F16, torch.bfloat16: B.BF16}[x.dtype]
+    dense_bytes = n * s
+    cap = B.cdma_zvc_max_compressed_bytes(n, code)
+    entries = B.cdma_zvc_table_entries(n)
+    ws_bytes = B.cdma_zvc_workspace_bytes(n, code)
+    payload = torch.empty(cap, dtype=torch.uint8, device=dev)
+    table = torch.empty(entries, dtype=torch.int64, device=dev)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    out = torch.empty_like(x)
+    res = torch.zeros(2, dtype=torch.int64).pin_memory()
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+
+    def compress():
+        st = B.cdma_zvc_compress_async(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap,
+                                       table.data_ptr(), ws.data_ptr(), ws_bytes, sh, res.data_ptr())
+        if st != B.OK:
+            raise B.CdmaError(st, "cdma_zvc_compress_async")
+
+    def decompress(c):
+        st = B.cdma_zvc_decompress_async(payload.data_ptr(), c, table.data_ptr(), n, code, B.NCHW,
+                                         out.data_ptr(), ws.data_ptr(), ws_bytes, sh, res.data_ptr())
+        if st != B.OK:
+            raise B.CdmaError(st, "cdma_zvc_decompress_async")
+
+    # ---- correctness on these very buffers before any timing ----------------
+    itype = torch.int32 if s == 4 else torch.int16
+    nnz = int(torch.count_nonzero(x.view(-1).view(itype)))
+    c_bytes = B.cdma_zvc_compress(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
+                                  ws.data_ptr(), ws_bytes, sh)
+    if c_bytes != 4 * ((n + 31) // 32) + s * nnz:
+        raise SystemExit("compressed size %d differs from 4*ceil(n/32)+s*nnz" % c_bytes)
+    r = B.cdma_zvc_decompress(payload.data_ptr(), c_bytes, table.data_ptr(), n, code, B.NCHW, out.data_ptr(),
+                              ws.data_ptr(), ws_bytes, sh)
+    if r != dense_bytes or not torch.equal(out.view(-1).view(itype), x.view(-1).view(itype)):
+        raise SystemExit("round trip is not bit-exact")
+    table_bytes = 8 * entries
+    algo_bytes = dense_bytes + c_bytes + table_bytes      # per kernel launch, either direction
+
+    # ---- device-resident timing --------------------------------------------
+    K, W = args.steps, max(args.warmup, 3)
+    for _ in range(W):
+        compress()
+        decompress(c_bytes)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K + 1)]
+    sampler = ClockSampler(local)
+    launches0 = B.cdma_kernel_launch_count()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev[0].record(stream)
+    for i in range(K):
+        compress()
+        ev[2 * i + 1].record(stream)
+        decompress(c_bytes)
+        ev[2 * i + 2].record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    launches = B.cdma_kernel_launch_count() - launches0
+    total_ms = ev[0].elapsed_time(ev[-1])
+    tc = [ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(K)]
+    td = [ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(K)]
+    if int(res[1]) != 0:
+        raise SystemExit("device reported status %d during timing" % int(res[1]))
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # ---- end to end with host buffers (copies inside the timed region) ------
+    e2e = None
+    offload = None
+    if not args.no_e2e:
+        e2e, offload = run_e2e(B, x, code, c_bytes, args, world, dev)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    mean_c, mean_d = sum(tc) / K, sum(td) / K
+
+    def roof(name, ms):
+        ach = algo_bytes / (ms * 1e-3) / 1e9
+        f = NCU_TRAFFIC_FACTOR.get(name)
+        return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+                "frac": ach / peak, "peak_kind": "of " + peak_kind,
+                "frac_of_nominal_8TBps": ach / NOMINAL_HBM_GBS,
+                "traffic": (f * algo_bytes) if f else None,
+                "algorithmic_bytes": algo_bytes, "mean_launch_ms": ms,
+                "uncompressed_GBps": dense_bytes / (ms * 1e-3) / 1e9}
+
+    rc, rd = roof("zvc_compress_kernel", mean_c), roof("zvc_decompress_kernel", mean_d)
+    dominant = rc if mean_c >= mean_d else rd
+    line = {
+        "metric": METRIC,
+        "value": world * dense_bytes * K / (total_ms * 1e-3) / 1e9,
+        "unit": UNIT,
+        "n_gpus": world,
+        "steps": K,
+        "warmup": W,
+        "ms_per_step": total_ms / K,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "u32" if s == 4 else "u16",
+        "data": "synthetic",
+        "config": {"workload": desc, "elements": n, "dense_bytes": dense_bytes,
+                   "compressed_bytes": c_bytes, "table_bytes": table_bytes,
+                   "density": nnz / n, "ratio_payload": dense_bytes / c_bytes,
+                   "ratio_with_table": dense_bytes / (c_bytes + table_bytes),
+                   "l2": "inputs larger than L2 (no flush needed)" if dense_bytes > 2 * 126e6
+                         else "input fits in L2: warm-cache figure",
+                   "parallelism": "replicas x%d, no collective" % world},
+        "roofline": dominant,
+        "kernels": {"compress": rc, "decompress": rd},
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+        "e2e": e2e,
+        "offload": offload,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        host = x.view(-1)[: min(n, 1 << 28)].cpu().numpy()
+        line["cpu_baseline"] = cpu_baseline(host)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(B, x, code, c_bytes, args, world, dev):
+    """The same round trip through the host-buffer entry points: dense tensor in
+    pinned host memory -> device -> compress -> payload in pinned host memory,
+    and back.  Also the natural offload/prefetch path (dense stays on the device,
+    only compressed bytes cross the link) against a plain pinned copy."""
+    import torch
+    import torch.distributed as dist
+    n, s = x.numel(), x.element_size()
+    dense_bytes = n * s
+    cap = B.cdma_zvc_max_compressed_bytes(n, code)
+    entries = B.cdma_zvc_table_entries(n)
+    staging = 2 * (cap + 8 * entries + B.cdma_zvc_workspace_bytes(n, code) + 4096)
+    ctx = B.cdma_ctx_create(cap + 8 * entries + 4096, staging)
+    h_x = torch.empty(x.shape, dtype=x.dtype).pin_memory()
+    h_x.copy_(x)
+    h_y = torch.empty(x.shape, dtype=x.dtype).pin_memory()
+    h_p = torch.empty(cap, dtype=torch.uint8).pin_memory()
+    h_t = torch.empty(entries, dtype=torch.int64).pin_memory()
+    steps = max(1, min(args.steps, args.e2e_steps))
+
+    def one():
+        c = B.cdma_zvc_compress_host(ctx, h_x.data_ptr(), n, code, B.NCHW, h_p.data_ptr(), cap, h_t.data_ptr())
+        if c != c_bytes:
+            raise SystemExit("host-buffer compress returned %d, expected %d" % (c, c_bytes))
+        r = B.cdma_zvc_decompress_host(ctx, h_p.data_ptr(), c, h_t.data_ptr(), n, code, B.NCHW, h_y.data_ptr())
+        if r != dense_bytes:
+            raise SystemExit("host-buffer decompress returned %d" % r)
+
+    one()
+    itype = torch.int32 if s == 4 else torch.int16
+    if not torch.equal(h_y.view(-1).view(itype), h_x.view(-1).view(itype)):
+        raise SystemExit("host-buffer round trip is not bit-exact")
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([dt], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+    e2e = {"value": world * dense_bytes * steps / dt / 1e9, "unit": UNIT,
+           "h2d_bytes_per_step": dense_bytes + c_bytes + 8 * entries,
+           "d2h_bytes_per_step": dense_bytes + c_bytes + 8 * entries,
+           "steps": steps, "ms_per_step": 1e3 * dt / steps,
+           "path": "cdma_zvc_compress_host + cdma_zvc_decompress_host on pinned host buffers"}
+
+    # natural path: OFF then PRE of the device tensor; only compressed bytes cross the link
+    stream = torch.cuda.current_stream()
+    out = torch.empty_like(x)
+
+    def off_pre():
+        c, t = B.cdma_offload(ctx, x.data_ptr(), n, code, B.NCHW, stream.cuda_stream)
+        if c != c_bytes:
+            raise SystemExit("cdma_offload returned %d" % c)
+        r = B.cdma_prefetch(ctx, t, out.data_ptr(), stream.cuda_stream)
+        if r != dense_bytes:
+            raise SystemExit("cdma_prefetch returned %d" % r)
+
+    off_pre()
+    if not torch.equal(out.view(-1).view(itype), x.view(-1).view(itype)):
+        raise SystemExit("offload/prefetch round trip is not bit-exact")
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        off_pre()
+    B.cdma_ctx_synchronize(ctx)
+    torch.cuda.synchronize()
+    dt_off = (time.perf_counter() - t0) / steps
+
+    # the uncompressed copy the compressed one replaces (pinned, both directions)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        h_y.copy_(x, non_blocking=True)
+        torch.cuda.synchronize()
+        out.copy_(h_y, non_blocking=True)
+        torch.cuda.synchronize()
+    dt_raw = (time.perf_counter() - t0) / steps
+    offload = {
+        "offload_prefetch_GBps": dense_bytes / dt_off / 1e9,
+        "plain_copy_round_trip_GBps": dense_bytes / dt_raw / 1e9,
+        "speedup_over_plain_copy": dt_raw / dt_off,
+        "pcie_round_trip_GBps_per_direction": 2 * dense_bytes / dt_raw / 1e9,
+        "link_bytes_per_step": 2 * (c_bytes + 8 * entries),
+        "note": "cdma_offload + cdma_prefetch per step vs pinned cudaMemcpy D2H + H2D of the dense tensor",
+    }
+    B.cdma_ctx_destroy(ctx)
+    return e2e, offload
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cdma", choices=["cdma", "reference"])
+    ap.add_argument("--workload", default="config2")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.steps < 1:
+        raise SystemExit("--steps must be >= 1")
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cdma(args)
+
+
+if __name__ == "__main__":
+    main()

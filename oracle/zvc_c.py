@@ -140,3 +140,25 @@ def check_table(payload: np.ndarray, n: int, s: int, table: np.ndarray) -> bool:
     if table.size != table_entries(n):
         return False
     return lib.zvc_oracle_check_table(_ptr(payload), payload.size, n, s, _ptr(table)) == 0
+
+
+def compress_into(x: np.ndarray, dst: np.ndarray, table: np.ndarray, threads: int = 1) -> int:
+    """Compress into caller-provided buffers (no allocation inside the timed call).
+    Returns the payload size or a negative error code."""
+    lib = _load()
+    raw = _as_bytes_view(x)
+    s = x.dtype.itemsize
+    if threads <= 1:
+        return int(lib.zvc_oracle_compress(_ptr(raw), x.size, s, _ptr(dst), dst.size, _ptr(table)))
+    return int(lib.zvc_oracle_compress_mt(_ptr(raw), x.size, s, _ptr(dst), dst.size, _ptr(table), threads))
+
+
+def decompress_into(payload: np.ndarray, table: np.ndarray, out: np.ndarray, threads: int = 1) -> int:
+    """Expand into a caller-provided array.  Returns bytes written or a negative error."""
+    lib = _load()
+    s = out.dtype.itemsize
+    outb = out.reshape(-1).view(np.uint8)
+    if threads <= 1:
+        return int(lib.zvc_oracle_decompress(_ptr(payload), payload.size, out.size, s, _ptr(outb)))
+    return int(lib.zvc_oracle_decompress_mt(_ptr(payload), payload.size, _ptr(table), out.size, s,
+                                            _ptr(outb), threads))
