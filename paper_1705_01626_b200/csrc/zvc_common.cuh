@@ -16,7 +16,7 @@ constexpr uint32_t kChunkWindows = 32;
 constexpr uint32_t kChunk = kWindow * kChunkWindows;   // 1024 elements
 
 // Compression tiling: one CTA = one tile = kTileChunks chunks, one warp per chunk.
-constexpr uint32_t kTileChunks = 8;
+constexpr uint32_t kTileChunks = 16;
 constexpr uint32_t kTileThreads = 32 * kTileChunks;
 
 // Workspace layout, in uint64 words.

@@ -2,15 +2,24 @@
 // prefix-sum / shift / append stages of the engine in Section V-B, Fig. 10a).
 //
 // One CTA compresses one tile of kTileChunks chunks; one warp owns one chunk
-// (32 windows of 32 elements).  Lane = element: a warp load of 32 consecutive
-// elements is one window, __ballot_sync of "bit pattern != 0" is its mask,
-// __popc of the mask below a lane is that element's slot among the window's
-// non-zeros.  Record sizes are scanned inside the warp and the CTA; the
-// running byte offset across tiles comes from a single-pass decoupled
-// look-back over 64-bit {state,value} descriptors, in ticket order so that a
-// tile only ever waits for tiles that are already running.  The tile's records
-// are assembled in shared memory at the same 16-byte phase as their place in
-// the payload and written out with 16-byte stores.
+// (32 windows of 32 elements).  A lane loads 4 consecutive elements with one
+// vector load, so a warp instruction covers 4 windows (8 lanes per window).
+//
+// Order of work inside a CTA, chosen so that the one step that depends on other
+// CTAs (the running byte offset across tiles) waits as little as possible:
+//   1. count: the tile's size needs only the number of non-zeros, so each warp
+//      reduces the pop-count of its "non-zero" nibbles and the tile's size is
+//      published at once, before any record exists;
+//   2. assemble: the 4-bit nibbles of the 8 lanes of a window are OR-combined
+//      with xor-shuffles into the window's 32-bit mask; __popc of the mask bits
+//      below a lane's nibble is the slot of its first value; records go to the
+//      warp's staging area in shared memory;
+//   3. look back: warp 0 walks the 64-bit {state,value} descriptors of earlier
+//      tiles (single-pass decoupled look-back, 32 per round), in ticket order
+//      so that a tile only ever waits for tiles that are already running; by
+//      now its predecessors have had the whole of step 2 to publish;
+//   4. copy: each warp writes its chunk's bytes to their place in the payload
+//      with coalesced stores.
 #include "zvc_common.cuh"
 
 namespace cdma {
@@ -22,20 +31,15 @@ struct LookbackResult {
     bool failed;
 };
 
-// Warp-wide look-back executed by warp 0 of the CTA.  Every lane inspects one
-// predecessor per round.  Waiting is bounded: when the limit is hit the tile
-// marks itself failed so that every later tile stops waiting too.
-__device__ LookbackResult decoupled_lookback(uint64_t* desc, uint64_t* ws, uint32_t tile,
-                                             uint64_t aggregate) {
+// Warp-wide walk executed by warp 0 of the CTA: lane l inspects tile look - l;
+// aggregates are added until a tile that already knows its inclusive prefix is
+// met.  Waiting for a predecessor that has not published yet is bounded: when
+// the limit is hit the tile marks itself failed so that every later tile stops
+// waiting too.
+__device__ LookbackResult lookback_walk(const uint64_t* desc, uint64_t* ws, uint32_t tile) {
     const uint32_t lane = lane_id();
     LookbackResult r{0, false};
-    if (tile == 0) {
-        if (lane == 0) st_relaxed_u64(desc, kDescPrefix | aggregate);
-        return r;
-    }
-    if (lane == 0) st_relaxed_u64(desc + tile, kDescAggregate | aggregate);
-
-    int64_t look = static_cast<int64_t>(tile) - 1;   // lane l inspects tile look - l
+    int64_t look = static_cast<int64_t>(tile) - 1;   // nearest tile not yet added
     uint32_t polls = 0;
     uint64_t t_start = 0;
     while (true) {
@@ -43,58 +47,71 @@ __device__ LookbackResult decoupled_lookback(uint64_t* desc, uint64_t* ws, uint3
         // before tile 0 there is nothing: an inclusive prefix of zero
         const uint64_t d = (idx >= 0) ? ld_relaxed_u64(desc + idx) : kDescPrefix;
         const uint32_t state = static_cast<uint32_t>(d >> 62);
-        const uint32_t is_invalid = __ballot_sync(0xffffffffu, state == 0);
-        const uint32_t is_prefix = __ballot_sync(0xffffffffu, state == 2);
-        const uint32_t is_error = __ballot_sync(0xffffffffu, state == 3);
-        // lanes up to and including the nearest tile that already knows its prefix
-        const uint32_t first = is_prefix & (0u - is_prefix);
-        const uint32_t upto = is_prefix ? (first | (first - 1u)) : 0xffffffffu;
-        if (is_error & upto) {
+        const uint32_t m_prefix = __ballot_sync(0xffffffffu, state == 2);
+        const uint32_t m_invalid = __ballot_sync(0xffffffffu, state == 0);
+        const uint32_t m_error = __ballot_sync(0xffffffffu, state == 3);
+        // lanes up to and including the nearest tile that knows its prefix
+        const uint32_t f = m_prefix & (0u - m_prefix);
+        const uint32_t upto = m_prefix ? (f | (f - 1u)) : 0xffffffffu;
+        if (m_error & upto) {
             r.failed = true;
             break;
         }
-        if (is_invalid & upto) {
-            if (polls == 0) t_start = global_timer_ns();
+        if (m_invalid & upto) {
             ++polls;
-            if (polls > kWaitLimitPolls || (global_timer_ns() - t_start) > kWaitLimitNs) {
-                if (lane == 0) report_status(ws, CDMA_ERR_TIMEOUT);
-                r.failed = true;
-                break;
+            if ((polls & 63u) == 0) {
+                const uint64_t now = global_timer_ns();
+                if (t_start == 0) t_start = now;
+                else if (now - t_start > kWaitLimitNs || polls > kWaitLimitPolls) {
+                    if (lane == 0) report_status(ws, CDMA_ERR_TIMEOUT);
+                    r.failed = true;
+                    break;
+                }
             }
-            __nanosleep(polls < 16 ? 32 : 256);
+            if (polls > 2) __nanosleep(100);
             continue;
         }
         uint64_t v = ((upto >> lane) & 1u) ? (d & kDescValueMask) : 0ull;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
         r.exclusive += v;
-        if (is_prefix) break;
+        if (m_prefix) break;
         look -= 32;
-    }
-    if (lane == 0) {
-        st_relaxed_u64(desc + tile, r.failed ? kDescError
-                                             : (kDescPrefix | (r.exclusive + aggregate)));
     }
     return r;
 }
 
+// Four consecutive elements as zero-extended 32-bit values.
+__device__ __forceinline__ void load4(const uint32_t* p, uint32_t (&e)[4]) {
+    const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
+    e[0] = q.x; e[1] = q.y; e[2] = q.z; e[3] = q.w;
+}
+__device__ __forceinline__ void load4(const uint16_t* p, uint32_t (&e)[4]) {
+    const uint2 q = __ldcs(reinterpret_cast<const uint2*>(p));
+    e[0] = q.x & 0xffffu; e[1] = q.x >> 16; e[2] = q.y & 0xffffu; e[3] = q.y >> 16;
+}
+
 template <typename T>
-__global__ void __launch_bounds__(kTileThreads)
+__global__ void __launch_bounds__(kTileThreads, 2)
 zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
                     uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
                     uint64_t num_chunks) {
     constexpr uint32_t S = sizeof(T);
-    constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
-    __shared__ __align__(16) uint8_t stage[kTileChunks * kMaxChunkBytes + 16];
+    constexpr uint32_t MU = 4 / S;                              // units of T per mask
+    constexpr uint32_t kMaxChunkUnits = MU * kChunkWindows + kChunk;
+    constexpr uint32_t kGroups = kChunk / 128;                  // 128 elements per warp load
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    T (*stage)[kMaxChunkUnits] = reinterpret_cast<T (*)[kMaxChunkUnits]>(smem_raw);
     __shared__ uint32_t s_tile;
-    __shared__ uint32_t s_chunk_bytes[kTileChunks];
+    __shared__ uint32_t s_chunk_units[kTileChunks];
     __shared__ uint32_t s_chunk_off[kTileChunks];
-    __shared__ uint32_t s_tile_bytes;
     __shared__ uint64_t s_base;
     __shared__ uint32_t s_failed;
 
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
+    const uint32_t sub = lane & 7u;       // position of this lane's nibble in its window
+    const uint32_t wj = lane >> 3;        // which of the 4 windows of a group
     uint64_t* desc = ws + kWsDescriptors;
 
     // Tiles are handed out in the order CTAs start running.
@@ -103,119 +120,139 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     const uint32_t tile = s_tile;
     if (tile >= num_tiles) return;
 
-    // ---- load: 32 windows of this warp's chunk, lane = element -------------
+    // ---- load the warp's chunk: 8 vector loads per lane, all in flight ------
     const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunks + warp;
     const uint64_t e0 = chunk * kChunk;
     uint32_t nwin;   // windows this chunk really has
-    T v[kChunkWindows];
+    uint32_t e[kGroups][4];
     if (e0 + kChunk <= n) {
         nwin = kChunkWindows;
-        const T* p = src + e0 + lane;
+        const T* p = src + e0 + 4 * lane;
 #pragma unroll
-        for (uint32_t w = 0; w < kChunkWindows; ++w) v[w] = __ldcs(p + w * kWindow);
+        for (uint32_t g = 0; g < kGroups; ++g) load4(p + g * 128, e[g]);
     } else {
         const uint64_t left = (e0 < n) ? (n - e0) : 0;
         nwin = static_cast<uint32_t>((left + kWindow - 1) / kWindow);
 #pragma unroll
-        for (uint32_t w = 0; w < kChunkWindows; ++w) {
-            const uint64_t j = static_cast<uint64_t>(w) * kWindow + lane;
-            v[w] = (j < left) ? __ldcs(src + e0 + j) : T(0);
+        for (uint32_t g = 0; g < kGroups; ++g) {
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) {
+                const uint64_t j = static_cast<uint64_t>(g) * 128 + 4 * lane + k;
+                e[g][k] = (j < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j)) : 0u;
+            }
         }
     }
 
-    // ---- masks: lane w keeps the mask of window w ---------------------------
-    uint32_t my_mask = 0;
+    // ---- 1. count: 4 "non-zero" bits per group, 8 groups packed in one word --
+    uint32_t nibs = 0;
 #pragma unroll
-    for (uint32_t w = 0; w < kChunkWindows; ++w) {
-        const uint32_t m = __ballot_sync(0xffffffffu, v[w] != T(0));
-        if (lane == w) my_mask = m;
+    for (uint32_t g = 0; g < kGroups; ++g) {
+        const uint32_t nib = (e[g][0] != 0u ? 1u : 0u) | (e[g][1] != 0u ? 2u : 0u) |
+                             (e[g][2] != 0u ? 4u : 0u) | (e[g][3] != 0u ? 8u : 0u);
+        nibs |= nib << (4 * g);
     }
-
-    // ---- record sizes and their exclusive scan inside the chunk -------------
-    const uint32_t my_rec = (lane < nwin) ? (4u + S * __popc(my_mask)) : 0u;
-    uint32_t incl = my_rec;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= static_cast<uint32_t>(o)) incl += t;
-    }
-    const uint32_t my_off = incl - my_rec;
-    if (lane == 31) s_chunk_bytes[warp] = incl;
+    const uint32_t units = MU * nwin + __reduce_add_sync(0xffffffffu, __popc(nibs));
+    if (lane == 0) s_chunk_units[warp] = units;
     __syncthreads();
-
-    // ---- chunk offsets inside the tile, then the tile's place in the stream -
+    uint64_t tile_bytes = 0;
     if (warp == 0) {
-        const uint32_t cb = (lane < kTileChunks) ? s_chunk_bytes[lane] : 0u;
-        uint32_t ci = cb;
+        const uint32_t cu = (lane < kTileChunks) ? s_chunk_units[lane] : 0u;
+        uint32_t ci = cu;
 #pragma unroll
         for (int o = 1; o < static_cast<int>(kTileChunks); o <<= 1) {
             const uint32_t t = __shfl_up_sync(0xffffffffu, ci, o);
             if (lane >= static_cast<uint32_t>(o)) ci += t;
         }
-        if (lane < kTileChunks) s_chunk_off[lane] = ci - cb;
-        const uint32_t tile_bytes = __shfl_sync(0xffffffffu, ci, kTileChunks - 1);
-        const LookbackResult lb = decoupled_lookback(desc, ws, tile, tile_bytes);
+        if (lane < kTileChunks) s_chunk_off[lane] = ci - cu;
+        tile_bytes = static_cast<uint64_t>(__shfl_sync(0xffffffffu, ci, kTileChunks - 1)) * S;
+        // the tile's size is public before any record is assembled
+        if (lane == 0)
+            st_relaxed_u64(desc + tile, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+    }
+
+    // ---- 2. assemble the chunk's records in shared memory --------------------
+    T* st = stage[warp];
+    uint32_t run = 0;                     // units of T emitted so far by this chunk
+    const uint32_t below = (1u << (4 * sub)) - 1u;
+#pragma unroll
+    for (uint32_t g = 0; g < kGroups; ++g) {
+        const uint32_t nib = (nibs >> (4 * g)) & 15u;
+        uint32_t m = nib << (4 * sub);
+        m |= __shfl_xor_sync(0xffffffffu, m, 1);
+        m |= __shfl_xor_sync(0xffffffffu, m, 2);
+        m |= __shfl_xor_sync(0xffffffffu, m, 4);               // the window's 32-bit mask
+        const bool live = (g * 4 + wj) < nwin;
+        const uint32_t rec = live ? (MU + __popc(m)) : 0u;     // record length, same in 8 lanes
+        uint32_t incl = rec;
+        uint32_t t = __shfl_up_sync(0xffffffffu, incl, 8);
+        if (lane >= 8) incl += t;
+        t = __shfl_up_sync(0xffffffffu, incl, 16);
+        if (lane >= 16) incl += t;                             // records of windows <= wj
+        const uint32_t pos = run + incl - rec;                 // where this window's record starts
+        run += __shfl_sync(0xffffffffu, incl, 31);
+        if (live) {
+            if (sub == 0) {
+                if (S == 4) {
+                    st[pos] = static_cast<T>(m);
+                } else {
+                    st[pos] = static_cast<T>(m & 0xffffu);
+                    st[pos + 1] = static_cast<T>(m >> 16);
+                }
+            }
+            uint32_t q = pos + MU + __popc(m & below);
+            if (nib & 1u) st[q++] = static_cast<T>(e[g][0]);
+            if (nib & 2u) st[q++] = static_cast<T>(e[g][1]);
+            if (nib & 4u) st[q++] = static_cast<T>(e[g][2]);
+            if (nib & 8u) st[q] = static_cast<T>(e[g][3]);
+        }
+    }
+
+    // ---- 3. the tile's place in the stream ------------------------------------
+    if (warp == 0) {
+        LookbackResult lb{0, false};
+        if (tile != 0) {
+            lb = lookback_walk(desc, ws, tile);
+            if (lane == 0)
+                st_relaxed_u64(desc + tile, lb.failed ? kDescError
+                                                      : (kDescPrefix | (lb.exclusive + tile_bytes)));
+        }
         if (lane == 0) {
-            s_tile_bytes = tile_bytes;
             s_base = lb.exclusive;
             s_failed = lb.failed ? 1u : 0u;
+            if (!lb.failed) {
+                if (tile == num_tiles - 1) {
+                    table[num_chunks] = lb.exclusive + tile_bytes;
+                    ws[kWsBytes] = lb.exclusive + tile_bytes;
+                }
+                if (lb.exclusive + tile_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
+            }
         }
     }
     __syncthreads();
     if (s_failed) return;
 
-    const uint64_t base = s_base;
-    const uint32_t tile_bytes = s_tile_bytes;
-    const uint32_t chunk_off = s_chunk_off[warp];
+    // ---- 4. each warp writes its chunk's bytes to their place, below cap ------
+    const uint64_t first_unit = s_base / S + s_chunk_off[warp];
+    if (lane == 0 && chunk < num_chunks) table[chunk] = first_unit * S;
+    const uint64_t cap_units = cap / S;
+    T* out = reinterpret_cast<T*>(dst) + first_unit;
+    const uint32_t room = (first_unit >= cap_units) ? 0u
+                        : (cap_units - first_unit < run ? static_cast<uint32_t>(cap_units - first_unit) : run);
+    for (uint32_t i = lane; i < room; i += 32) out[i] = st[i];
+}
 
-    if (lane == 0 && chunk < num_chunks) table[chunk] = base + chunk_off;
-    if (tile == num_tiles - 1 && threadIdx.x == 0) {
-        table[num_chunks] = base + tile_bytes;
-        ws[kWsBytes] = base + tile_bytes;
-    }
-    if (threadIdx.x == 0 && base + tile_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
-
-    // ---- assemble the records in shared memory ------------------------------
-    // Byte b of the tile's output sits at stage[phase + b], phase = base mod 16,
-    // so that 16-byte groups of the payload are 16-byte groups of `stage`.
-    const uint32_t phase = static_cast<uint32_t>(base & 15u);
-    T* out = reinterpret_cast<T*>(stage + phase + chunk_off);   // S divides every offset
-    const uint32_t lt = lanemask_lt();
-#pragma unroll
-    for (uint32_t w = 0; w < kChunkWindows; ++w) {
-        const uint32_t m = __shfl_sync(0xffffffffu, my_mask, w);
-        const uint32_t off = __shfl_sync(0xffffffffu, my_off, w) / S;
-        if (w < nwin) {
-            if (S == 4) {
-                if (lane == 0) out[off] = static_cast<T>(m);
-            } else {
-                if (lane < 2) out[off + lane] = static_cast<T>(m >> (16 * lane));
-            }
-            if ((m >> lane) & 1u) out[off + 4 / S + __popc(m & lt)] = v[w];
-        }
-    }
-    __syncthreads();
-
-    // ---- write the tile's bytes [base, base + tile_bytes) below cap ---------
-    const uint64_t g0 = base;
-    const uint64_t g1 = (base + tile_bytes < cap) ? (base + tile_bytes) : cap;
-    if (g0 >= g1) return;
-    const uint64_t a0 = g0 & ~15ull;                 // stage[0] corresponds to payload byte a0
-    const uint32_t nvec = static_cast<uint32_t>((g1 - a0 + 15) >> 4);
-    for (uint32_t i = threadIdx.x; i < nvec; i += kTileThreads) {
-        const uint64_t ga = a0 + 16ull * i;
-        if (ga >= g0 && ga + 16 <= g1) {
-            __stcs(reinterpret_cast<uint4*>(dst + ga), *reinterpret_cast<const uint4*>(stage + 16u * i));
-        } else {
-            // ragged edge of the tile: element-sized stores, clipped to [g0, g1)
-#pragma unroll
-            for (uint32_t b = 0; b < 16; b += S) {
-                const uint64_t gb = ga + b;
-                if (gb >= g0 && gb < g1)
-                    *reinterpret_cast<T*>(dst + gb) = *reinterpret_cast<const T*>(stage + 16u * i + b);
-            }
-        }
-    }
+template <typename T>
+cudaError_t launch_typed(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
+                         uint64_t* d_ws, cudaStream_t stream) {
+    constexpr uint32_t kSmem = kTileChunks * (4 * kChunkWindows + sizeof(T) * kChunk);
+    const cudaError_t e = cudaFuncSetAttribute(zvc_compress_kernel<T>,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    const uint64_t tiles = num_tiles_of(n);
+    zvc_compress_kernel<T><<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
+        static_cast<const T*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
+        static_cast<uint32_t>(tiles), num_chunks_of(n));
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -223,21 +260,12 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
 cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst,
                                 uint64_t cap, uint64_t* d_table, uint64_t* d_ws,
                                 cudaStream_t stream) {
-    const uint64_t chunks = num_chunks_of(n);
-    const uint64_t tiles = num_tiles_of(n);
-    if (tiles == 0) return cudaSuccess;
-    const dim3 grid(static_cast<unsigned>(tiles));
-    if (elem_size == 4) {
-        zvc_compress_kernel<uint32_t><<<grid, kTileThreads, 0, stream>>>(
-            static_cast<const uint32_t*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
-            static_cast<uint32_t>(tiles), chunks);
-    } else {
-        zvc_compress_kernel<uint16_t><<<grid, kTileThreads, 0, stream>>>(
-            static_cast<const uint16_t*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
-            static_cast<uint32_t>(tiles), chunks);
-    }
+    if (num_tiles_of(n) == 0) return cudaSuccess;
+    const cudaError_t e = (elem_size == 4)
+                              ? launch_typed<uint32_t>(d_src, n, d_dst, cap, d_table, d_ws, stream)
+                              : launch_typed<uint16_t>(d_src, n, d_dst, cap, d_table, d_ws, stream);
     count_kernel_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace cdma

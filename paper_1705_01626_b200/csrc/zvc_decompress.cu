@@ -6,11 +6,13 @@
 // chunk's byte range in the payload; the warp copies that range into shared
 // memory with 16-byte loads, then walks the records: the position of window
 // w+1's mask is the position of window w's mask plus 4 plus s times the
-// pop-count of that mask (the stream is self-delimiting, Section V-A).  Lane =
-// element: a lane whose mask bit is set reads the value at its rank among the
-// set bits below it, the others write zero; every window is one coalesced
-// store.  The table and every record are validated; nothing is read outside
-// the payload or written outside the tensor whatever the input holds.
+// pop-count of that mask (the stream is self-delimiting, Section V-A).  A lane
+// expands 4 consecutive elements, so one warp store covers 4 windows (8 lanes
+// per window): the lane takes its 4 mask bits, the pop-count of the mask bits
+// below them is where its first value sits, it reads 4 candidate values and
+// selects value-or-zero for each element, then stores them as one vector.
+// The table and every record are validated; nothing is read outside the
+// payload or written outside the tensor whatever the input holds.
 #include "zvc_common.cuh"
 
 namespace cdma {
@@ -20,14 +22,24 @@ namespace {
 constexpr uint32_t kDecWarps = 8;
 constexpr uint32_t kDecThreads = 32 * kDecWarps;
 
+__device__ __forceinline__ void store4(uint32_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(a, b, c, d));
+}
+__device__ __forceinline__ void store4(uint16_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    __stcs(reinterpret_cast<uint2*>(p), make_uint2(a | (b << 16), c | (d << 16)));
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kDecThreads)
 zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
                       const uint64_t* __restrict__ table, uint64_t n, T* __restrict__ dst,
                       uint64_t* __restrict__ ws, uint64_t num_chunks) {
     constexpr uint32_t S = sizeof(T);
+    constexpr uint32_t MU = 4 / S;                               // units of T per mask
     constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
-    constexpr uint32_t kBuf = kMaxChunkBytes + 32;   // 16-byte phase in front, round-up behind
+    // 16-byte phase in front; behind, room for the reads of a walk that has
+    // left a malformed record (clamped to `end`, then at most a mask and 35 values)
+    constexpr uint32_t kBuf = kMaxChunkBytes + 16 + 160;
     __shared__ __align__(16) uint8_t s_buf[kDecWarps][kBuf];
 
     const uint32_t lane = lane_id();
@@ -79,22 +91,56 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
     const T* units = reinterpret_cast<const T*>(buf);
     uint32_t p = static_cast<uint32_t>(lo - a0) / S;        // position in units of S bytes
     const uint32_t end = static_cast<uint32_t>(hi - a0) / S;
-    const uint32_t lt = lanemask_lt();
     bool bad = false;
-    T* out = dst + e0 + lane;
-#pragma unroll 8
-    for (uint32_t w = 0; w < nwin; ++w) {
-        if (p + 4 / S > end) { bad = true; break; }
-        uint32_t m;
-        if (S == 4) m = units[p];
-        else m = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
-        const uint32_t cnt = __popc(m);
-        const uint32_t left = nelem - w * kWindow;           // elements this window really has
-        if (p + 4 / S + cnt > end || (left < kWindow && (m >> left) != 0)) { bad = true; break; }
-        const bool bit = (m >> lane) & 1u;
-        const T val = bit ? units[p + 4 / S + __popc(m & lt)] : T(0);
-        if (lane < left) __stcs(out + w * kWindow, val);
-        p += 4 / S + cnt;
+
+    if (nelem == kChunk) {
+        // full chunk: 8 rounds of 4 windows; lane = 4 consecutive elements
+        const uint32_t sub = lane & 7u;
+        const uint32_t wj = lane >> 3;
+        const uint32_t below = (1u << (4 * sub)) - 1u;
+        T* out = dst + e0 + 4 * lane;
+#pragma unroll
+        for (uint32_t g = 0; g < kChunk / 128; ++g) {
+            uint32_t my_p = 0, my_m = 0;
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j) {
+                uint32_t m;
+                if (S == 4) m = units[p];
+                else m = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
+                if (wj == j) { my_p = p; my_m = m; }
+                p += MU + __popc(m);
+                bad |= (p > end);
+                p = min(p, end);                  // a malformed record cannot drag reads away
+            }
+            const uint32_t nib = (my_m >> (4 * sub)) & 15u;
+            const uint32_t q = my_p + MU + __popc(my_m & below);
+            const uint32_t a = units[q], b = units[q + 1], c = units[q + 2], d = units[q + 3];
+            // element k takes the candidate numbered by the set bits below bit k
+            const uint32_t v0 = (nib & 1u) ? a : 0u;
+            const uint32_t v1 = (nib & 2u) ? ((nib & 1u) ? b : a) : 0u;
+            const uint32_t c2 = __popc(nib & 3u);
+            const uint32_t v2 = (nib & 4u) ? (c2 == 0 ? a : (c2 == 1 ? b : c)) : 0u;
+            const uint32_t c3 = __popc(nib & 7u);
+            const uint32_t v3 = (nib & 8u) ? (c3 == 0 ? a : (c3 == 1 ? b : (c3 == 2 ? c : d))) : 0u;
+            store4(out + g * 128, v0, v1, v2, v3);
+        }
+    } else {
+        // ragged last chunk: lane = element, one window per round
+        const uint32_t lt = lanemask_lt();
+        T* out = dst + e0 + lane;
+        for (uint32_t w = 0; w < nwin; ++w) {
+            if (p + MU > end) { bad = true; break; }
+            uint32_t m;
+            if (S == 4) m = units[p];
+            else m = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
+            const uint32_t cnt = __popc(m);
+            const uint32_t left = nelem - w * kWindow;           // elements this window really has
+            if (p + MU + cnt > end || (left < kWindow && (m >> left) != 0)) { bad = true; break; }
+            const bool bit = (m >> lane) & 1u;
+            const T val = bit ? units[p + MU + __popc(m & lt)] : T(0);
+            if (lane < left) out[w * kWindow] = val;
+            p += MU + cnt;
+        }
     }
     if (!bad && p != end) bad = true;
     if (bad && lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
