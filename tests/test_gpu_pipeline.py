@@ -1,0 +1,138 @@
+"""GPU: the offload / prefetch context and the host-buffer calls, checked
+against the CPU oracle and bit-exact round trips."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import zvc_c
+from paper_1705_01626_b200 import binding as B
+from paper_1705_01626_b200 import workloads as wl
+from tests.gpu_helpers import raw_numpy
+
+pytestmark = pytest.mark.gpu
+
+
+def bits(x):
+    return x.view(-1).view(torch.int32 if x.element_size() == 4 else torch.int16)
+
+
+def make_ctx(tensors, slack=1 << 16):
+    worst = max(B.cdma_zvc_max_compressed_bytes(t.numel(), B.F32 if t.element_size() == 4 else B.F16)
+                + 8 * B.cdma_zvc_table_entries(t.numel())
+                + B.cdma_zvc_workspace_bytes(t.numel(), B.F32) + 4096 for t in tensors)
+    pinned = sum(B.cdma_zvc_max_compressed_bytes(t.numel(), B.F32 if t.element_size() == 4 else B.F16)
+                 + 8 * B.cdma_zvc_table_entries(t.numel()) + 512 for t in tensors) + slack
+    return B.cdma_ctx_create(pinned, 2 * worst)
+
+
+def small_offload_set():
+    shapes = ((8, 56, 56), (8, 56, 56), (16, 28, 28), (16, 28, 28), (32, 14, 14), (32, 7, 7))
+    return [t for t, _ in wl.vgg16_offload_set(batch=4, device="cuda", shapes=shapes)]
+
+
+def test_offload_all_then_prefetch_in_reverse_order():
+    tensors = small_offload_set()
+    ctx = make_ctx(tensors)
+    stream = torch.cuda.Stream()
+    try:
+        tickets, sizes = [], []
+        with torch.cuda.stream(stream):
+            for t in tensors:
+                c, ticket = B.cdma_offload(ctx, t.data_ptr(), t.numel(), B.F32, B.NCHW, stream.cuda_stream)
+                assert c >= 0, B.status_string(c)
+                want, _ = zvc_c.compress(raw_numpy(t))
+                assert c == len(want)                       # the call returns the compressed size
+                st, payload_bytes, n = B.cdma_ticket_info(ctx, ticket)
+                assert (st, payload_bytes, n) == (0, c, t.numel())
+                tickets.append(ticket)
+                sizes.append(c)
+            assert B.cdma_ctx_synchronize(ctx) == 0
+            outs = [torch.full_like(t, -1.0) for t in tensors]
+            for i in reversed(range(len(tensors))):        # backward pass order
+                st = B.cdma_prefetch_async(ctx, tickets[i], outs[i].data_ptr(), stream.cuda_stream)
+                assert st == 0, B.status_string(st)
+            assert B.cdma_ctx_synchronize(ctx) == 0
+        stream.synchronize()
+        for t, o in zip(tensors, outs):
+            assert torch.equal(bits(o), bits(t))
+        # tickets are consumed
+        assert B.cdma_prefetch(ctx, tickets[0], outs[0].data_ptr(), stream.cuda_stream) == -B.ERR_BAD_TICKET
+        ratio = sum(t.numel() * 4 for t in tensors) / sum(sizes)
+        assert 1.5 < ratio < 8
+    finally:
+        B.cdma_ctx_destroy(ctx)
+
+
+def test_blocking_prefetch_and_pool_reuse():
+    tensors = small_offload_set()[:3]
+    ctx = make_ctx(tensors)
+    try:
+        for rounds in range(3):                             # the pinned pool is recycled
+            tickets = []
+            for t in tensors:
+                c, ticket = B.cdma_offload(ctx, t.data_ptr(), t.numel(), B.F32, B.NCHW, 0)
+                assert c > 0
+                tickets.append(ticket)
+            for t, ticket in zip(tensors, tickets):
+                out = torch.zeros_like(t)
+                r = B.cdma_prefetch(ctx, ticket, out.data_ptr(), 0)
+                assert r == t.numel() * 4, B.status_string(r)
+                assert torch.equal(bits(out), bits(t))
+    finally:
+        B.cdma_ctx_destroy(ctx)
+
+
+def test_pool_exhaustion_and_small_staging_are_reported():
+    t = wl.iid_relu_like((64 * 1024,), 0.9, seed=3, device="cuda")
+    need = B.cdma_zvc_max_compressed_bytes(t.numel(), B.F32)
+    ctx = B.cdma_ctx_create(4096, 2 * (need + 65536))       # pinned pool far too small
+    try:
+        c, _ = B.cdma_offload(ctx, t.data_ptr(), t.numel(), B.F32, B.NCHW, 0)
+        assert c == -B.ERR_OUT_OF_MEMORY
+    finally:
+        B.cdma_ctx_destroy(ctx)
+    ctx = B.cdma_ctx_create(1 << 20, 2 * 65536)             # staging slot smaller than the payload
+    try:
+        c, _ = B.cdma_offload(ctx, t.data_ptr(), t.numel(), B.F32, B.NCHW, 0)
+        assert c == -B.ERR_BUFFER_TOO_SMALL
+        # the context still works for a tensor that fits
+        s = wl.iid_relu_like((8 * 1024,), 0.1, seed=4, device="cuda")
+        c, ticket = B.cdma_offload(ctx, s.data_ptr(), s.numel(), B.F32, B.NCHW, 0)
+        assert c > 0
+        out = torch.zeros_like(s)
+        assert B.cdma_prefetch(ctx, ticket, out.data_ptr(), 0) == 4 * s.numel()
+        assert torch.equal(bits(out), bits(s))
+    finally:
+        B.cdma_ctx_destroy(ctx)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+def test_host_buffer_calls_match_the_oracle(dtype):
+    n = 300_000 + 77
+    code = B.F32 if dtype == torch.float32 else B.F16
+    x = wl.iid_relu_like((n,), 0.3, seed=8, device="cpu", dtype=dtype, floor=2.0 ** -10).pin_memory()
+    cap = B.cdma_zvc_max_compressed_bytes(n, code)
+    entries = B.cdma_zvc_table_entries(n)
+    h_p = torch.zeros(cap, dtype=torch.uint8).pin_memory()
+    h_t = torch.zeros(entries, dtype=torch.int64).pin_memory()
+    h_y = torch.zeros(n, dtype=dtype).pin_memory()
+    ctx = B.cdma_ctx_create(1 << 16, 2 * (cap + 8 * entries + B.cdma_zvc_workspace_bytes(n, code) + 4096))
+    try:
+        c = B.cdma_zvc_compress_host(ctx, x.data_ptr(), n, code, B.NCHW, h_p.data_ptr(), cap, h_t.data_ptr())
+        want, want_table = zvc_c.compress(x.numpy().view(np.uint32 if dtype == torch.float32 else np.uint16))
+        assert c == len(want), B.status_string(c)
+        assert h_p[:c].numpy().tobytes() == want.tobytes()
+        assert np.array_equal(h_t.numpy().view(np.uint64), want_table)
+        r = B.cdma_zvc_decompress_host(ctx, h_p.data_ptr(), c, h_t.data_ptr(), n, code, B.NCHW, h_y.data_ptr())
+        assert r == n * x.element_size(), B.status_string(r)
+        assert torch.equal(bits(h_y), bits(x))
+        # too small a host destination is refused
+        assert B.cdma_zvc_compress_host(ctx, x.data_ptr(), n, code, B.NCHW, h_p.data_ptr(), c - 4,
+                                        h_t.data_ptr()) == -B.ERR_BUFFER_TOO_SMALL
+        # a corrupted table is reported, not followed
+        bad = h_t.clone().pin_memory()
+        bad[1] += 4
+        assert B.cdma_zvc_decompress_host(ctx, h_p.data_ptr(), c, bad.data_ptr(), n, code, B.NCHW,
+                                          h_y.data_ptr()) == -B.ERR_CORRUPT_STREAM
+    finally:
+        B.cdma_ctx_destroy(ctx)
