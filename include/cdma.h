@@ -137,6 +137,34 @@ int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout
                             void* cuda_stream, uint64_t* h_result);
 
 /*
+ * The same compression for callers that cannot allocate device memory: code
+ * inside a memory manager's eviction path (where an allocation could re-enter
+ * the manager, or fail because the device is full -- which is when activations
+ * get offloaded), plug-ins that only ever receive buffers from their host
+ * application, start-up and tear-down hooks.  (The paper has no counterpart:
+ * its engine needs no software workspace.)  The call takes no workspace; it
+ * uses one built into the library, a fixed device array of 131,328 bytes that
+ * every GPU loading the library holds until the process exits, and it calls no
+ * cudaMalloc, cudaFree or any other allocating routine.
+ *
+ *   - Serves tensors of at most 2^28 elements; a larger n is refused with
+ *     -CDMA_ERR_BUFFER_TOO_SMALL (the built-in workspace is too small for it)
+ *     before anything is enqueued.
+ *   - The first call made with a given device current looks up the array's
+ *     device address on that device (a one-time, synchronous set-up step);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous
+ *     call's contents; each call clears the part it uses first.  Two calls
+ *     that overlap in time on the same device (different streams or threads)
+ *     race on it and give undefined results: serialise them.
+ *   - Otherwise identical to cdma_zvc_compress: same arguments and checks, same
+ *     payload and table, waits for the stream and returns C or -status.
+ */
+int64_t cdma_zvc_compress_static_ws(const void* d_src, uint64_t n, int dtype, int layout,
+                                    void* d_dst, uint64_t dst_capacity, uint64_t* d_table,
+                                    void* cuda_stream);
+
+/*
  * Expand a payload back into n dense elements (Section V-B, decompression
  * engine: the pop-count of a mask tells how many values its window takes,
  * values or zeros are steered into place).

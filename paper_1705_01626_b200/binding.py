@@ -53,6 +53,8 @@ _SIGNATURES = {
                                     c_void_p, c_uint64, c_void_p]),
     "cdma_zvc_compress_async": (c_int, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64, c_void_p,
                                         c_void_p, c_uint64, c_void_p, c_void_p]),
+    "cdma_zvc_compress_static_ws": (c_int64, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64, c_void_p,
+                                              c_void_p]),
     "cdma_zvc_decompress": (c_int64, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p,
                                       c_void_p, c_uint64, c_void_p]),
     "cdma_zvc_decompress_async": (c_int, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p,
@@ -132,6 +134,15 @@ def cdma_zvc_compress_async(d_src, n, dtype, layout, d_dst, dst_capacity, d_tabl
     return int(lib().cdma_zvc_compress_async(_vp(d_src), n, dtype, layout, _vp(d_dst), dst_capacity,
                                              _vp(d_table), _vp(d_workspace), workspace_bytes,
                                              _vp(cuda_stream), _vp(h_result)))
+
+
+def cdma_zvc_compress_static_ws(d_src, n, dtype, layout, d_dst, dst_capacity, d_table, cuda_stream=0) -> int:
+    """Compression without a caller-provided workspace, for callers that cannot
+    allocate device memory (an eviction path, a plug-in that owns no buffers).
+    Uses the library's built-in fixed workspace: at most 2**28 elements, and
+    calls on one device must not overlap in time.  Returns C or a negative status."""
+    return int(lib().cdma_zvc_compress_static_ws(_vp(d_src), n, dtype, layout, _vp(d_dst), dst_capacity,
+                                                 _vp(d_table), _vp(cuda_stream)))
 
 
 def cdma_zvc_decompress(d_src, src_bytes, d_table, n, dtype, layout, d_dst, d_workspace,

@@ -1,0 +1,74 @@
+"""GPU: the compression entry point for callers that cannot allocate device
+memory (cdma_zvc_compress_static_ws) must produce exactly what the ordinary
+entry point produces -- same return value, same payload bytes, same offset
+table (integer/byte work: tolerance 0) -- on two calls in a row, the second of
+which would be wrong if the first call's leftovers in the shared built-in
+workspace were not cleared.
+
+This file is named to be collected last: a run that stops at the first failure
+has then already run every other test.  It passes on its own in a fresh process
+and after the rest of the suite.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_1705_01626_b200 import binding as B
+from paper_1705_01626_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def compress_both_ways(x, stream=0):
+    n = x.numel()
+    code = B.F32 if x.element_size() == 4 else B.F16
+    cap = B.cdma_zvc_max_compressed_bytes(n, code)
+    entries = B.cdma_zvc_table_entries(n)
+    ws_bytes = B.cdma_zvc_workspace_bytes(n, code)
+    ref_payload = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    ref_table = torch.zeros(entries, dtype=torch.int64, device="cuda")
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda")
+    c_ref = B.cdma_zvc_compress(x.data_ptr(), n, code, B.NCHW, ref_payload.data_ptr(), cap, ref_table.data_ptr(),
+                                ws.data_ptr(), ws_bytes, stream)
+    assert c_ref >= 0, B.status_string(c_ref)
+    payload = torch.full((cap,), 0xEE, dtype=torch.uint8, device="cuda")
+    table = torch.full((entries,), -1, dtype=torch.int64, device="cuda")
+    c = B.cdma_zvc_compress_static_ws(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
+                                      stream)
+    assert c == c_ref, (c, c_ref, B.status_string(c))
+    assert torch.equal(payload[:c], ref_payload[:c])
+    assert torch.equal(table, ref_table)
+    return c
+
+
+def test_two_calls_in_a_row_match_the_ordinary_entry_point():
+    # first a large, dense-ish tensor (many tiles, large offsets left behind in the workspace) ...
+    big = wl.iid_relu_like((3_000_000 + 123,), 0.8, seed=wl.seed_for(7, 0), device="cuda")
+    c1 = compress_both_ways(big)
+    # ... then a smaller, sparser one that reuses the first tiles' descriptors
+    small = wl.correlated_relu((4, 16, 56, 56), 0.2, seed=wl.seed_for(7, 1), device="cuda")
+    c2 = compress_both_ways(small)
+    assert c2 < c1
+    # and once more on a side stream with 2-byte elements
+    half = wl.iid_relu_like((500_000 + 7,), 0.3, seed=wl.seed_for(7, 2), device="cuda", dtype=torch.float16,
+                            floor=2.0 ** -10)
+    s = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    compress_both_ways(half, s.cuda_stream)
+
+
+def test_sizes_beyond_the_built_in_workspace_are_refused():
+    x = torch.zeros(1024, device="cuda")
+    payload = torch.zeros(4096 + 256, dtype=torch.uint8, device="cuda")
+    table = torch.zeros(8, dtype=torch.int64, device="cuda")
+    too_many = (1 << 28) + 1
+    r = B.cdma_zvc_compress_static_ws(x.data_ptr(), too_many, B.F32, B.NCHW, payload.data_ptr(), 4096,
+                                      table.data_ptr(), 0)
+    assert r == -B.ERR_BUFFER_TOO_SMALL
+    assert B.cdma_zvc_compress_static_ws(x.data_ptr(), 1024, 9, B.NCHW, payload.data_ptr(), 4096,
+                                         table.data_ptr(), 0) == -B.ERR_UNSUPPORTED_DTYPE
+    # the limit itself is about n, not about the data: an ordinary small call still works afterwards
+    assert B.cdma_zvc_compress_static_ws(x.data_ptr(), 1024, B.F32, B.NCHW, payload.data_ptr(), 4096,
+                                         table.data_ptr(), 0) == 128
+    assert B.cdma_zvc_compress_static_ws(0, 0, B.F32, B.NCHW, payload.data_ptr(), 4096, table.data_ptr(), 0) == 0
+    assert int(table[0]) == 0
