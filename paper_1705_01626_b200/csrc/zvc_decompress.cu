@@ -37,9 +37,12 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
     constexpr uint32_t S = sizeof(T);
     constexpr uint32_t MU = 4 / S;                               // units of T per mask
     constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
-    // 16-byte phase in front; behind, room for the reads of a walk that has
-    // left a malformed record (clamped to `end`, then at most a mask and 35 values)
-    constexpr uint32_t kBuf = kMaxChunkBytes + 16 + 160;
+    // 16-byte phase in front; behind, room for the reads of a walk that has left
+    // a malformed record: it is pulled back to `end` after every group of 4
+    // windows, so it can run at most 4 records (4*(MU+32) units) past `end`, and
+    // a lane then reads a mask and up to 35 values from there
+    constexpr uint32_t kBuf = (kMaxChunkBytes + 16 + S * (4 * (MU + 32) + MU + 36) + 15) / 16 * 16;
+    static_assert(kBuf % 16 == 0, "rows of s_buf must keep 16-byte alignment for the vector stores");
     __shared__ __align__(16) uint8_t s_buf[kDecWarps][kBuf];
 
     const uint32_t lane = lane_id();
@@ -101,28 +104,28 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
         T* out = dst + e0 + 4 * lane;
 #pragma unroll
         for (uint32_t g = 0; g < kChunk / 128; ++g) {
-            uint32_t my_p = 0, my_m = 0;
+            // four serial steps of the self-delimiting walk; every lane sees all four
+            uint32_t pw[4], mw[4];
 #pragma unroll
             for (uint32_t j = 0; j < 4; ++j) {
-                uint32_t m;
-                if (S == 4) m = units[p];
-                else m = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
-                if (wj == j) { my_p = p; my_m = m; }
-                p += MU + __popc(m);
-                bad |= (p > end);
-                p = min(p, end);                  // a malformed record cannot drag reads away
+                pw[j] = p;
+                if (S == 4) mw[j] = units[p];
+                else mw[j] = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
+                p += MU + __popc(mw[j]);
             }
+            // a malformed record may have carried the walk past the chunk: flag it and
+            // pull the position back so that no later read leaves the staged bytes
+            bad |= (p > end);
+            p = min(p, end);
+            const uint32_t my_p = (wj == 0) ? pw[0] : (wj == 1) ? pw[1] : (wj == 2) ? pw[2] : pw[3];
+            const uint32_t my_m = (wj == 0) ? mw[0] : (wj == 1) ? mw[1] : (wj == 2) ? mw[2] : mw[3];
             const uint32_t nib = (my_m >> (4 * sub)) & 15u;
             const uint32_t q = my_p + MU + __popc(my_m & below);
-            const uint32_t a = units[q], b = units[q + 1], c = units[q + 2], d = units[q + 3];
-            // element k takes the candidate numbered by the set bits below bit k
-            const uint32_t v0 = (nib & 1u) ? a : 0u;
-            const uint32_t v1 = (nib & 2u) ? ((nib & 1u) ? b : a) : 0u;
-            const uint32_t c2 = __popc(nib & 3u);
-            const uint32_t v2 = (nib & 4u) ? (c2 == 0 ? a : (c2 == 1 ? b : c)) : 0u;
-            const uint32_t c3 = __popc(nib & 7u);
-            const uint32_t v3 = (nib & 8u) ? (c3 == 0 ? a : (c3 == 1 ? b : (c3 == 2 ? c : d))) : 0u;
-            store4(out + g * 128, v0, v1, v2, v3);
+            // element k takes the value numbered by the set bits below bit k
+            const uint32_t c1 = nib & 1u, c2 = __popc(nib & 3u), c3 = __popc(nib & 7u);
+            const uint32_t a0v = units[q], a1v = units[q + c1], a2v = units[q + c2], a3v = units[q + c3];
+            store4(out + g * 128, (nib & 1u) ? a0v : 0u, (nib & 2u) ? a1v : 0u, (nib & 4u) ? a2v : 0u,
+                   (nib & 8u) ? a3v : 0u);
         }
     } else {
         // ragged last chunk: lane = element, one window per round
