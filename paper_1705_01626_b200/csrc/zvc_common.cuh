@@ -16,11 +16,11 @@ constexpr uint32_t kChunkWindows = 32;
 constexpr uint32_t kChunk = kWindow * kChunkWindows;   // 1024 elements
 
 // Compression tiling: one CTA = one tile = kTileChunks chunks, one warp per chunk.
-constexpr uint32_t kTileChunks = 16;
+constexpr uint32_t kTileChunks = 12;
 constexpr uint32_t kTileThreads = 32 * kTileChunks;
 
 // Workspace layout, in uint64 words.
-constexpr uint32_t kWsTicket = 0;      // next tile ticket (low 32 bits)
+constexpr uint32_t kWsTicket = 0;      // reserved (tiles are taken in block-index order)
 constexpr uint32_t kWsReserved = 1;
 constexpr uint32_t kWsBytes = 2;       // result: payload bytes (compress) / dense bytes (decompress)
 constexpr uint32_t kWsStatus = 3;      // result: first error code, 0 = none

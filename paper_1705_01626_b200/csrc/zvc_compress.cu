@@ -15,9 +15,9 @@
 //      below a lane's nibble is the slot of its first value; records go to the
 //      warp's staging area in shared memory;
 //   3. look back: warp 0 walks the 64-bit {state,value} descriptors of earlier
-//      tiles (single-pass decoupled look-back, 32 per round), in ticket order
-//      so that a tile only ever waits for tiles that are already running; by
-//      now its predecessors have had the whole of step 2 to publish;
+//      tiles (single-pass decoupled look-back, 32 per round); tiles follow the
+//      block index, so a tile only ever waits for blocks dispatched before it;
+//      by now its predecessors have had the whole of step 2 to publish;
 //   4. copy: each warp writes its chunk's bytes to their place in the payload
 //      with coalesced stores.
 #include "zvc_common.cuh"
@@ -92,7 +92,7 @@ __device__ __forceinline__ void load4(const uint16_t* p, uint32_t (&e)[4]) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kTileThreads, 2)
+__global__ void __launch_bounds__(kTileThreads, 3)
 zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
                     uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
                     uint64_t num_chunks) {
@@ -102,7 +102,6 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     constexpr uint32_t kGroups = kChunk / 128;                  // 128 elements per warp load
     extern __shared__ __align__(16) uint8_t smem_raw[];
     T (*stage)[kMaxChunkUnits] = reinterpret_cast<T (*)[kMaxChunkUnits]>(smem_raw);
-    __shared__ uint32_t s_tile;
     __shared__ uint32_t s_chunk_units[kTileChunks];
     __shared__ uint32_t s_chunk_off[kTileChunks];
     __shared__ uint64_t s_base;
@@ -114,10 +113,11 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     const uint32_t wj = lane >> 3;        // which of the 4 windows of a group
     uint64_t* desc = ws + kWsDescriptors;
 
-    // Tiles are handed out in the order CTAs start running.
-    if (threadIdx.x == 0) s_tile = atomicAdd(reinterpret_cast<unsigned int*>(ws + kWsTicket), 1u);
-    __syncthreads();
-    const uint32_t tile = s_tile;
+    // Tile = block index.  Thread blocks are dispatched in increasing index order,
+    // so every tile this one will wait for belongs to a block that is already
+    // running or finished (the assumption single-pass scans rest on); should it
+    // ever not hold, the bounded wait below turns it into CDMA_ERR_TIMEOUT.
+    const uint32_t tile = blockIdx.x;
     if (tile >= num_tiles) return;
 
     // ---- load the warp's chunk: 8 vector loads per lane, all in flight ------
