@@ -241,17 +241,189 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     for (uint32_t i = lane; i < room; i += 32) out[i] = st[i];
 }
 
-template <typename T>
-cudaError_t launch_typed(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
-                         uint64_t* d_ws, cudaStream_t stream) {
-    constexpr uint32_t kSmem = kTileChunks * (4 * kChunkWindows + sizeof(T) * kChunk);
-    const cudaError_t e = cudaFuncSetAttribute(zvc_compress_kernel<T>,
-                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+// 2-byte elements: the same four steps with 8 consecutive elements per lane (one
+// 16-byte load), so a warp instruction covers 8 windows (4 lanes per window), and
+// two chunks per warp, so that a tile is as many bytes (48 KB) as in the 4-byte
+// kernel and the look-back runs at the same rate per byte.
+constexpr uint32_t kTileChunksU16 = 2 * kTileChunks;
+
+__global__ void __launch_bounds__(kTileThreads, 3)
+zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst,
+                        uint64_t cap, uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
+                        uint32_t num_tiles, uint64_t num_chunks) {
+    using T = uint16_t;
+    constexpr uint32_t S = 2, MU = 2;
+    constexpr uint32_t kMaxChunkUnits = MU * kChunkWindows + kChunk;
+    constexpr uint32_t kGroups = kChunk / 256;                  // 256 elements per warp load
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    T (*stage)[kMaxChunkUnits] = reinterpret_cast<T (*)[kMaxChunkUnits]>(smem_raw);
+    __shared__ uint32_t s_chunk_units[kTileChunksU16];
+    __shared__ uint32_t s_chunk_off[kTileChunksU16];
+    __shared__ uint64_t s_base;
+    __shared__ uint32_t s_failed;
+
+    const uint32_t lane = lane_id();
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint32_t sub = lane & 3u;       // position of this lane's byte in its window's mask
+    const uint32_t wj = lane >> 2;        // which of the 8 windows of a group
+    uint64_t* desc = ws + kWsDescriptors;
+    const uint32_t tile = blockIdx.x;     // block-index order, as in the 4-byte kernel
+    if (tile >= num_tiles) return;
+
+    // ---- load the warp's two chunks ------------------------------------------
+    uint32_t nwin[2];
+    uint32_t w[2][kGroups][4];            // 8 elements of a group = 4 words of two halves
+#pragma unroll
+    for (uint32_t c = 0; c < 2; ++c) {
+        const uint64_t e0 = (static_cast<uint64_t>(tile) * kTileChunksU16 + 2 * warp + c) * kChunk;
+        if (e0 + kChunk <= n) {
+            nwin[c] = kChunkWindows;
+            const T* p = src + e0 + 8 * lane;
+#pragma unroll
+            for (uint32_t g = 0; g < kGroups; ++g) {
+                const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p + g * 256));
+                w[c][g][0] = q.x; w[c][g][1] = q.y; w[c][g][2] = q.z; w[c][g][3] = q.w;
+            }
+        } else {
+            const uint64_t left = (e0 < n) ? (n - e0) : 0;
+            nwin[c] = static_cast<uint32_t>((left + kWindow - 1) / kWindow);
+#pragma unroll
+            for (uint32_t g = 0; g < kGroups; ++g) {
+#pragma unroll
+                for (uint32_t k = 0; k < 4; ++k) {
+                    const uint64_t j = static_cast<uint64_t>(g) * 256 + 8 * lane + 2 * k;
+                    const uint32_t lo = (j < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j)) : 0u;
+                    const uint32_t hi = (j + 1 < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j + 1)) : 0u;
+                    w[c][g][k] = lo | (hi << 16);
+                }
+            }
+        }
+    }
+
+    // ---- 1. count: 8 "non-zero" bits per group, 4 groups packed in one word --
+    uint32_t bits[2];
+#pragma unroll
+    for (uint32_t c = 0; c < 2; ++c) {
+        bits[c] = 0;
+#pragma unroll
+        for (uint32_t g = 0; g < kGroups; ++g) {
+            uint32_t b8 = 0;
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) {
+                b8 |= ((w[c][g][k] & 0xffffu) != 0u ? 1u : 0u) << (2 * k);
+                b8 |= ((w[c][g][k] >> 16) != 0u ? 2u : 0u) << (2 * k);
+            }
+            bits[c] |= b8 << (8 * g);
+        }
+        const uint32_t units = MU * nwin[c] + __reduce_add_sync(0xffffffffu, __popc(bits[c]));
+        if (lane == 0) s_chunk_units[2 * warp + c] = units;
+    }
+    __syncthreads();
+    uint64_t tile_bytes = 0;
+    if (warp == 0) {
+        const uint32_t cu = (lane < kTileChunksU16) ? s_chunk_units[lane] : 0u;
+        uint32_t ci = cu;
+#pragma unroll
+        for (int o = 1; o < static_cast<int>(kTileChunksU16); o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, ci, o);
+            if (lane >= static_cast<uint32_t>(o)) ci += t;
+        }
+        if (lane < kTileChunksU16) s_chunk_off[lane] = ci - cu;
+        tile_bytes = static_cast<uint64_t>(__shfl_sync(0xffffffffu, ci, kTileChunksU16 - 1)) * S;
+        if (lane == 0)
+            st_relaxed_u64(desc + tile, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+    }
+
+    // ---- 2. assemble the records of both chunks in shared memory -------------
+    uint32_t run[2];
+    const uint32_t below = (1u << (8 * sub)) - 1u;
+#pragma unroll
+    for (uint32_t c = 0; c < 2; ++c) {
+        T* st = stage[2 * warp + c];
+        uint32_t r = 0;
+#pragma unroll
+        for (uint32_t g = 0; g < kGroups; ++g) {
+            const uint32_t b8 = (bits[c] >> (8 * g)) & 0xffu;
+            uint32_t m = b8 << (8 * sub);
+            m |= __shfl_xor_sync(0xffffffffu, m, 1);
+            m |= __shfl_xor_sync(0xffffffffu, m, 2);           // the window's 32-bit mask
+            const bool live = (g * 8 + wj) < nwin[c];
+            const uint32_t rec = live ? (MU + __popc(m)) : 0u;
+            uint32_t incl = rec;
+            uint32_t t = __shfl_up_sync(0xffffffffu, incl, 4);
+            if (lane >= 4) incl += t;
+            t = __shfl_up_sync(0xffffffffu, incl, 8);
+            if (lane >= 8) incl += t;
+            t = __shfl_up_sync(0xffffffffu, incl, 16);
+            if (lane >= 16) incl += t;                         // records of windows <= wj
+            const uint32_t pos = r + incl - rec;
+            r += __shfl_sync(0xffffffffu, incl, 31);
+            if (live) {
+                if (sub == 0) {
+                    st[pos] = static_cast<T>(m & 0xffffu);
+                    st[pos + 1] = static_cast<T>(m >> 16);
+                }
+                uint32_t q = pos + MU + __popc(m & below);
+#pragma unroll
+                for (uint32_t k = 0; k < 4; ++k) {
+                    if (b8 & (1u << (2 * k))) st[q++] = static_cast<T>(w[c][g][k] & 0xffffu);
+                    if (b8 & (2u << (2 * k))) st[q++] = static_cast<T>(w[c][g][k] >> 16);
+                }
+            }
+        }
+        run[c] = r;
+    }
+
+    // ---- 3. the tile's place in the stream ------------------------------------
+    if (warp == 0) {
+        LookbackResult lb{0, false};
+        if (tile != 0) {
+            lb = lookback_walk(desc, ws, tile);
+            if (lane == 0)
+                st_relaxed_u64(desc + tile, lb.failed ? kDescError
+                                                      : (kDescPrefix | (lb.exclusive + tile_bytes)));
+        }
+        if (lane == 0) {
+            s_base = lb.exclusive;
+            s_failed = lb.failed ? 1u : 0u;
+            if (!lb.failed) {
+                if (tile == num_tiles - 1) {
+                    table[num_chunks] = lb.exclusive + tile_bytes;
+                    ws[kWsBytes] = lb.exclusive + tile_bytes;
+                }
+                if (lb.exclusive + tile_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
+            }
+        }
+    }
+    __syncthreads();
+    if (s_failed) return;
+
+    // ---- 4. each warp writes its chunks' bytes to their place, below cap ------
+    const uint64_t cap_units = cap / S;
+#pragma unroll
+    for (uint32_t c = 0; c < 2; ++c) {
+        const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunksU16 + 2 * warp + c;
+        const uint64_t first_unit = s_base / S + s_chunk_off[2 * warp + c];
+        if (lane == 0 && chunk < num_chunks) table[chunk] = first_unit * S;
+        T* out = reinterpret_cast<T*>(dst) + first_unit;
+        const T* st = stage[2 * warp + c];
+        const uint32_t room = (first_unit >= cap_units) ? 0u
+                            : (cap_units - first_unit < run[c] ? static_cast<uint32_t>(cap_units - first_unit) : run[c]);
+        for (uint32_t i = lane; i < room; i += 32) out[i] = st[i];
+    }
+}
+
+template <typename T, uint32_t TILE_CHUNKS, typename Kernel>
+cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_dst, uint64_t cap,
+                         uint64_t* d_table, uint64_t* d_ws, cudaStream_t stream) {
+    constexpr uint32_t kSmem = TILE_CHUNKS * (4 * kChunkWindows + sizeof(T) * kChunk);
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    const uint64_t tiles = num_tiles_of(n);
-    zvc_compress_kernel<T><<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
+    const uint64_t chunks = num_chunks_of(n);
+    const uint64_t tiles = (chunks + TILE_CHUNKS - 1) / TILE_CHUNKS;   // never more than num_tiles_of(n)
+    kernel<<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
         static_cast<const T*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
-        static_cast<uint32_t>(tiles), num_chunks_of(n));
+        static_cast<uint32_t>(tiles), chunks);
     return cudaGetLastError();
 }
 
@@ -261,9 +433,10 @@ cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_siz
                                 uint64_t cap, uint64_t* d_table, uint64_t* d_ws,
                                 cudaStream_t stream) {
     if (num_tiles_of(n) == 0) return cudaSuccess;
-    const cudaError_t e = (elem_size == 4)
-                              ? launch_typed<uint32_t>(d_src, n, d_dst, cap, d_table, d_ws, stream)
-                              : launch_typed<uint16_t>(d_src, n, d_dst, cap, d_table, d_ws, stream);
+    const cudaError_t e =
+        (elem_size == 4)
+            ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t>, d_src, n, d_dst, cap, d_table, d_ws, stream)
+            : launch_typed<uint16_t, kTileChunksU16>(zvc_compress_kernel_u16, d_src, n, d_dst, cap, d_table, d_ws, stream);
     count_kernel_launch();
     return e;
 }
