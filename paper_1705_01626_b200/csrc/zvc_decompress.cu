@@ -38,10 +38,14 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
     constexpr uint32_t MU = 4 / S;                               // units of T per mask
     constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
     // 16-byte phase in front; behind, room for the reads of a walk that has left
-    // a malformed record: it is pulled back to `end` after every group of 4
-    // windows, so it can run at most 4 records (4*(MU+32) units) past `end`, and
-    // a lane then reads a mask and up to 35 values from there
-    constexpr uint32_t kBuf = (kMaxChunkBytes + 16 + S * (4 * (MU + 32) + MU + 36) + 15) / 16 * 16;
+    // a malformed record.  4-byte elements: the position is pulled back to `end`
+    // after every window (one more instruction per window, but the smaller buffer
+    // lets a sixth CTA fit per SM); 2-byte elements: after every group of 4
+    // windows, so the walk can run 4 records past `end`.  Either way a lane then
+    // reads a mask and up to 35 values from there.
+    constexpr bool kClampEveryWindow = (S == 4);
+    constexpr uint32_t kOverrun = kClampEveryWindow ? 0u : 4u * (MU + 32u);
+    constexpr uint32_t kBuf = (kMaxChunkBytes + 16 + S * (kOverrun + MU + 36) + 15) / 16 * 16;
     static_assert(kBuf % 16 == 0, "rows of s_buf must keep 16-byte alignment for the vector stores");
     __shared__ __align__(16) uint8_t s_buf[kDecWarps][kBuf];
 
@@ -112,11 +116,11 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
                 if (S == 4) mw[j] = units[p];
                 else mw[j] = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
                 p += MU + __popc(mw[j]);
+                // a malformed record may carry the walk past the chunk: flag it and pull
+                // the position back so that no later read leaves the staged bytes
+                if (kClampEveryWindow) { bad |= (p > end); p = min(p, end); }
             }
-            // a malformed record may have carried the walk past the chunk: flag it and
-            // pull the position back so that no later read leaves the staged bytes
-            bad |= (p > end);
-            p = min(p, end);
+            if (!kClampEveryWindow) { bad |= (p > end); p = min(p, end); }
             const uint32_t my_p = (wj == 0) ? pw[0] : (wj == 1) ? pw[1] : (wj == 2) ? pw[2] : pw[3];
             const uint32_t my_m = (wj == 0) ? mw[0] : (wj == 1) ? mw[1] : (wj == 2) ? mw[2] : mw[3];
             const uint32_t nib = (my_m >> (4 * sub)) & 15u;
