@@ -242,12 +242,35 @@ int64_t cdma_offload(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, in
 int64_t cdma_prefetch(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream);
 int cdma_prefetch_async(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream);
 
+/*
+ * The same OFF / PRE with no device staging and no second copy, closest to the
+ * single compressed-copy call the paper envisions (Section V-D): the compress
+ * kernel stores its payload and table straight into the context's pinned pool
+ * (mapped into the device's address space), so the bytes cross the host link as
+ * the kernel produces them, and the decompress kernel loads them from there.
+ * Only the workspace is taken from a staging slot.  Both calls wait for their
+ * kernel -- which now lasts as long as the transfer -- and return C / n*s.
+ * cdma_offload_direct reserves the worst-case size in the pool while it runs
+ * and gives the unused part back; tickets of either kind can be prefetched by
+ * either cdma_prefetch or cdma_prefetch_direct.
+ */
+int64_t cdma_offload_direct(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, int layout,
+                            void* compute_stream, cdma_ticket* out);
+int64_t cdma_prefetch_direct(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream);
+
 /* Wait for everything the context enqueued; returns the first deferred
  * failure of an asynchronous call since the last synchronize, else 0. */
 int cdma_ctx_synchronize(cdma_ctx* ctx);
 
 /* Size facts of a live ticket: payload bytes and element count. 0 on success. */
 int cdma_ticket_info(cdma_ctx* ctx, cdma_ticket ticket, uint64_t* payload_bytes, uint64_t* n);
+
+/* Host pointers to a live ticket's payload (payload_bytes long, see
+ * cdma_ticket_info) and table inside the pinned pool, e.g. to write an offloaded
+ * activation map to storage.  Waits for pending copies into the pool.  The
+ * pointers stay valid until the ticket is prefetched or the context destroyed. */
+int cdma_ticket_host_view(cdma_ctx* ctx, cdma_ticket ticket, const void** h_payload,
+                          const uint64_t** h_table);
 
 /*
  * The same compressed copies for callers whose tensors live in HOST memory

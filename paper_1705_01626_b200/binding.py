@@ -64,8 +64,11 @@ _SIGNATURES = {
     "cdma_offload": (c_int64, [c_void_p, c_void_p, c_uint64, c_int, c_int, c_void_p, POINTER(cdma_ticket)]),
     "cdma_prefetch": (c_int64, [c_void_p, cdma_ticket, c_void_p, c_void_p]),
     "cdma_prefetch_async": (c_int, [c_void_p, cdma_ticket, c_void_p, c_void_p]),
+    "cdma_offload_direct": (c_int64, [c_void_p, c_void_p, c_uint64, c_int, c_int, c_void_p, POINTER(cdma_ticket)]),
+    "cdma_prefetch_direct": (c_int64, [c_void_p, cdma_ticket, c_void_p, c_void_p]),
     "cdma_ctx_synchronize": (c_int, [c_void_p]),
     "cdma_ticket_info": (c_int, [c_void_p, cdma_ticket, POINTER(c_uint64), POINTER(c_uint64)]),
+    "cdma_ticket_host_view": (c_int, [c_void_p, cdma_ticket, POINTER(c_void_p), POINTER(c_void_p)]),
     "cdma_zvc_compress_host": (c_int64, [c_void_p, c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64,
                                          c_void_p]),
     "cdma_zvc_decompress_host": (c_int64, [c_void_p, c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int,
@@ -187,6 +190,18 @@ def cdma_prefetch_async(ctx, ticket, d_dst, compute_stream=0) -> int:
     return int(lib().cdma_prefetch_async(ctx, ticket, _vp(d_dst), _vp(compute_stream)))
 
 
+def cdma_offload_direct(ctx, d_src, n, dtype, layout, compute_stream=0):
+    """Compress straight into the pinned pool (no staging, no second copy).  Returns (C or negative status, ticket)."""
+    t = cdma_ticket(0)
+    r = lib().cdma_offload_direct(ctx, _vp(d_src), n, dtype, layout, _vp(compute_stream), ctypes.byref(t))
+    return int(r), t
+
+
+def cdma_prefetch_direct(ctx, ticket, d_dst, compute_stream=0) -> int:
+    """Decompress straight from the pinned pool.  Returns n*s or a negative status."""
+    return int(lib().cdma_prefetch_direct(ctx, ticket, _vp(d_dst), _vp(compute_stream)))
+
+
 def cdma_ctx_synchronize(ctx) -> int:
     return int(lib().cdma_ctx_synchronize(ctx))
 
@@ -196,6 +211,13 @@ def cdma_ticket_info(ctx, ticket):
     c, n = c_uint64(0), c_uint64(0)
     st = lib().cdma_ticket_info(ctx, ticket, ctypes.byref(c), ctypes.byref(n))
     return int(st), int(c.value), int(n.value)
+
+
+def cdma_ticket_host_view(ctx, ticket):
+    """Returns (status, host address of the payload, host address of the table)."""
+    hp, ht = c_void_p(0), c_void_p(0)
+    st = lib().cdma_ticket_host_view(ctx, ticket, ctypes.byref(hp), ctypes.byref(ht))
+    return int(st), hp.value or 0, ht.value or 0
 
 
 def cdma_zvc_compress_host(ctx, h_src, n, dtype, layout, h_dst, dst_capacity, h_table) -> int:

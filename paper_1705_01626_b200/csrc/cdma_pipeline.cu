@@ -40,6 +40,12 @@ public:
         }
         return false;
     }
+    // Give back the tail of a region that turned out larger than needed.
+    void shrink(uint64_t off, uint64_t old_bytes, uint64_t new_bytes) {
+        old_bytes = round_up(old_bytes ? old_bytes : 1, kAlign);
+        new_bytes = round_up(new_bytes ? new_bytes : 1, kAlign);
+        if (new_bytes < old_bytes) release(off + new_bytes, old_bytes - new_bytes);
+    }
     void release(uint64_t off, uint64_t bytes) {
         bytes = round_up(bytes ? bytes : 1, kAlign);
         auto it = free_.emplace(off, bytes).first;
@@ -82,7 +88,8 @@ struct TicketRec {
     uint64_t n;
     int dtype, layout;
     uint64_t payload_bytes;
-    uint64_t pool_off, pool_bytes;
+    uint64_t pool_off, pool_bytes;      // region of the pinned pool owned by the ticket
+    uint64_t payload_off, table_off;    // where payload and table sit inside the pool
 };
 
 }  // namespace
@@ -176,7 +183,7 @@ int cdma_ctx_create(uint64_t pinned_bytes, uint64_t device_staging_bytes, cdma_c
             st = CDMA_ERR_CUDA; break;
         }
         if (pinned_bytes &&
-            cudaHostAlloc(reinterpret_cast<void**>(&ctx->h_pool), pinned_bytes, cudaHostAllocDefault) !=
+            cudaHostAlloc(reinterpret_cast<void**>(&ctx->h_pool), pinned_bytes, cudaHostAllocMapped | cudaHostAllocPortable) !=
                 cudaSuccess) {
             st = CDMA_ERR_OUT_OF_MEMORY; break;
         }
@@ -250,10 +257,12 @@ int64_t cdma_offload(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, in
 
     // exactly C payload bytes and the table cross the link (Section V-D: the
     // compressed size is known on completion and sizes the host allocation)
-    TicketRec rec{n, dtype, layout, c, 0, round_up(c, 16) + p.table_bytes};
+    TicketRec rec{n, dtype, layout, c, 0, round_up(c, 16) + p.table_bytes, 0, 0};
     if (!ctx->pool.alloc(rec.pool_bytes, &rec.pool_off) ||
         rec.pool_off + rec.pool_bytes > ctx->pool_bytes)
         return -static_cast<int64_t>(CDMA_ERR_OUT_OF_MEMORY);
+    rec.payload_off = rec.pool_off;
+    rec.table_off = rec.pool_off + round_up(c, 16);
     uint8_t* h = ctx->h_pool + rec.pool_off;
     bool ok = true;
     if (c) ok &= cudaMemcpyAsync(h, p.payload, c, cudaMemcpyDeviceToHost, ctx->side) == cudaSuccess;
@@ -284,13 +293,12 @@ static int prefetch_enqueue(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void
     if (!plan_slot(slot, rec.n, rec.dtype, &p) || p.capacity < rec.payload_bytes)
         return CDMA_ERR_BUFFER_TOO_SMALL;
     if (slot.used && cudaStreamWaitEvent(ctx->side, slot.idle, 0) != cudaSuccess) return CDMA_ERR_CUDA;
-    const uint8_t* h = ctx->h_pool + rec.pool_off;
     bool ok = true;
     if (rec.payload_bytes)
-        ok &= cudaMemcpyAsync(p.payload, h, rec.payload_bytes, cudaMemcpyHostToDevice, ctx->side) ==
-              cudaSuccess;
-    ok &= cudaMemcpyAsync(p.table, h + round_up(rec.payload_bytes, 16), p.table_bytes,
-                          cudaMemcpyHostToDevice, ctx->side) == cudaSuccess;
+        ok &= cudaMemcpyAsync(p.payload, ctx->h_pool + rec.payload_off, rec.payload_bytes,
+                              cudaMemcpyHostToDevice, ctx->side) == cudaSuccess;
+    ok &= cudaMemcpyAsync(p.table, ctx->h_pool + rec.table_off, p.table_bytes, cudaMemcpyHostToDevice,
+                          ctx->side) == cudaSuccess;
     ok &= cudaEventRecord(slot.staged, ctx->side) == cudaSuccess;
     ok &= cudaStreamWaitEvent(compute, slot.staged, 0) == cudaSuccess;
     if (!ok) return CDMA_ERR_CUDA;
@@ -331,6 +339,97 @@ int64_t cdma_prefetch(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* comp
     return static_cast<int64_t>(dense);
 }
 
+
+// ---- direct variants: the kernels read and write the pinned pool themselves ----------------------
+// (Section V-D: one call that compresses while it copies and reports the size on completion; here the
+// copy over the host link is the kernel's own stores into mapped host memory.)
+
+int64_t cdma_offload_direct(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, int layout,
+                            void* compute_stream, cdma_ticket* out) {
+    if (ctx == nullptr || out == nullptr) return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
+    if (cdma_dtype_size(dtype) == 0) return -static_cast<int64_t>(CDMA_ERR_UNSUPPORTED_DTYPE);
+    cudaStream_t compute = static_cast<cudaStream_t>(compute_stream);
+    // only the workspace lives on the device: take it from a staging slot
+    Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
+    const uint64_t ws_bytes = cdma_zvc_workspace_bytes(n, dtype);
+    if (slot.bytes < ws_bytes) return -static_cast<int64_t>(CDMA_ERR_BUFFER_TOO_SMALL);
+    // the size is unknown until the kernel is done: reserve the worst case, give the rest back after
+    const uint64_t table_bytes = 8 * cdma_zvc_table_entries(n);
+    const uint64_t cap = cdma_zvc_max_compressed_bytes(n, dtype);
+    TicketRec rec{n, dtype, layout, 0, 0, round_up(table_bytes, kAlign) + cap, 0, 0};
+    if (!ctx->pool.alloc(rec.pool_bytes, &rec.pool_off) || rec.pool_off + rec.pool_bytes > ctx->pool_bytes)
+        return -static_cast<int64_t>(CDMA_ERR_OUT_OF_MEMORY);
+    rec.table_off = rec.pool_off;
+    rec.payload_off = rec.pool_off + round_up(table_bytes, kAlign);
+    void* d_payload = nullptr;
+    void* d_table = nullptr;
+    if (cudaHostGetDevicePointer(&d_payload, ctx->h_pool + rec.payload_off, 0) != cudaSuccess ||
+        cudaHostGetDevicePointer(&d_table, ctx->h_pool + rec.table_off, 0) != cudaSuccess) {
+        cudaGetLastError();
+        ctx->pool.release(rec.pool_off, rec.pool_bytes);
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    }
+    if (slot.used && cudaStreamWaitEvent(compute, slot.idle, 0) != cudaSuccess) {
+        ctx->pool.release(rec.pool_off, rec.pool_bytes);
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    }
+    uint64_t* res = next_result_words(ctx);
+    const int st = cdma_zvc_compress_async(d_src, n, dtype, layout, d_payload, cap, static_cast<uint64_t*>(d_table),
+                                           slot.base, slot.bytes, compute, res);
+    if (st != CDMA_OK) {
+        ctx->pool.release(rec.pool_off, rec.pool_bytes);
+        return -static_cast<int64_t>(st);
+    }
+    slot.used = true;
+    if (cudaEventRecord(slot.idle, compute) != cudaSuccess || cudaEventSynchronize(slot.idle) != cudaSuccess) {
+        ctx->pool.release(rec.pool_off, rec.pool_bytes);
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    }
+    if (res[1] != 0) {
+        ctx->pool.release(rec.pool_off, rec.pool_bytes);
+        return -static_cast<int64_t>(res[1]);
+    }
+    rec.payload_bytes = res[0];
+    const uint64_t used = round_up(table_bytes, kAlign) + rec.payload_bytes;
+    ctx->pool.shrink(rec.pool_off, rec.pool_bytes, used);
+    rec.pool_bytes = used;
+    out->id = ctx->next_ticket++;
+    ctx->tickets[out->id] = rec;
+    return static_cast<int64_t>(rec.payload_bytes);
+}
+
+int64_t cdma_prefetch_direct(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream) {
+    if (ctx == nullptr) return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
+    auto it = ctx->tickets.find(ticket.id);
+    if (it == ctx->tickets.end()) return -static_cast<int64_t>(CDMA_ERR_BAD_TICKET);
+    const TicketRec rec = it->second;
+    cudaStream_t compute = static_cast<cudaStream_t>(compute_stream);
+    Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
+    if (slot.bytes < cdma_zvc_workspace_bytes(rec.n, rec.dtype)) return -static_cast<int64_t>(CDMA_ERR_BUFFER_TOO_SMALL);
+    void* d_payload = nullptr;
+    void* d_table = nullptr;
+    if (cudaHostGetDevicePointer(&d_payload, ctx->h_pool + rec.payload_off, 0) != cudaSuccess ||
+        cudaHostGetDevicePointer(&d_table, ctx->h_pool + rec.table_off, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    }
+    // earlier copies into this region were enqueued on the side stream: let them land first
+    if (cudaStreamSynchronize(ctx->side) != cudaSuccess) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (slot.used && cudaStreamWaitEvent(compute, slot.idle, 0) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    uint64_t* res = next_result_words(ctx);
+    const int st = cdma_zvc_decompress_async(d_payload, rec.payload_bytes, static_cast<const uint64_t*>(d_table), rec.n,
+                                             rec.dtype, rec.layout, d_dst, slot.base, slot.bytes, compute, res);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    slot.used = true;
+    if (cudaEventRecord(slot.idle, compute) != cudaSuccess || cudaEventSynchronize(slot.idle) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    ctx->pool.release(rec.pool_off, rec.pool_bytes);
+    ctx->tickets.erase(it);
+    if (res[1] != 0) return -static_cast<int64_t>(res[1]);
+    return static_cast<int64_t>(rec.n * cdma_dtype_size(rec.dtype));
+}
+
 int cdma_ctx_synchronize(cdma_ctx* ctx) {
     if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
     const int st = wait_all(ctx);
@@ -346,6 +445,17 @@ int cdma_ticket_info(cdma_ctx* ctx, cdma_ticket ticket, uint64_t* payload_bytes,
     if (it == ctx->tickets.end()) return CDMA_ERR_BAD_TICKET;
     if (payload_bytes) *payload_bytes = it->second.payload_bytes;
     if (n) *n = it->second.n;
+    return CDMA_OK;
+}
+
+int cdma_ticket_host_view(cdma_ctx* ctx, cdma_ticket ticket, const void** h_payload, const uint64_t** h_table) {
+    if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
+    auto it = ctx->tickets.find(ticket.id);
+    if (it == ctx->tickets.end()) return CDMA_ERR_BAD_TICKET;
+    // copies into the pool are asynchronous on the side stream: let them land before the host looks
+    if (cudaStreamSynchronize(ctx->side) != cudaSuccess) return CDMA_ERR_CUDA;
+    if (h_payload) *h_payload = ctx->h_pool + it->second.payload_off;
+    if (h_table) *h_table = reinterpret_cast<const uint64_t*>(ctx->h_pool + it->second.table_off);
     return CDMA_OK;
 }
 

@@ -1,5 +1,7 @@
 """GPU: the offload / prefetch context and the host-buffer calls, checked
 against the CPU oracle and bit-exact round trips."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -134,5 +136,59 @@ def test_host_buffer_calls_match_the_oracle(dtype):
         bad[1] += 4
         assert B.cdma_zvc_decompress_host(ctx, h_p.data_ptr(), c, bad.data_ptr(), n, code, B.NCHW,
                                           h_y.data_ptr()) == -B.ERR_CORRUPT_STREAM
+    finally:
+        B.cdma_ctx_destroy(ctx)
+
+
+def host_view(ctx, ticket, nbytes, entries):
+    st, hp, ht = B.cdma_ticket_host_view(ctx, ticket)
+    assert st == 0
+    payload = np.frombuffer(ctypes.string_at(hp, nbytes), dtype=np.uint8)
+    table = np.frombuffer(ctypes.string_at(ht, 8 * entries), dtype=np.uint64)
+    return payload, table
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+def test_direct_offload_writes_the_oracle_stream_into_the_pinned_pool(dtype):
+    code = B.F32 if dtype == torch.float32 else B.F16
+    tensors = [wl.iid_relu_like((n,), d, seed=31 + i, device="cuda", dtype=dtype, floor=2.0 ** -10)
+               for i, (n, d) in enumerate([(700_000 + 13, 0.3), (12 * 1024 * 5, 0.9), (1000, 0.0), (333_333, 0.05)])]
+    worst = max(B.cdma_zvc_max_compressed_bytes(t.numel(), code) + 8 * B.cdma_zvc_table_entries(t.numel()) + 4096
+                for t in tensors)
+    ctx = B.cdma_ctx_create(len(tensors) * worst + (1 << 16), 2 * (worst + (1 << 20)))
+    try:
+        tickets = []
+        for t in tensors:                                    # direct: kernel stores into host memory
+            c, tk = B.cdma_offload_direct(ctx, t.data_ptr(), t.numel(), code, B.NCHW, 0)
+            assert c >= 0, B.status_string(c)
+            want, want_table = zvc_c.compress(raw_numpy(t))
+            assert c == len(want)
+            got, got_table = host_view(ctx, tk, c, B.cdma_zvc_table_entries(t.numel()))
+            assert got.tobytes() == want.tobytes()
+            assert np.array_equal(got_table, want_table)
+            tickets.append(tk)
+        # staged tickets hold the same bytes
+        c2, tk2 = B.cdma_offload(ctx, tensors[0].data_ptr(), tensors[0].numel(), code, B.NCHW, 0)
+        got, got_table = host_view(ctx, tk2, c2, B.cdma_zvc_table_entries(tensors[0].numel()))
+        want, want_table = zvc_c.compress(raw_numpy(tensors[0]))
+        assert got.tobytes() == want.tobytes() and np.array_equal(got_table, want_table)
+        # either kind of ticket can come back either way
+        outs = [torch.full_like(t, 3.0) for t in tensors]
+        for i in reversed(range(len(tensors))):
+            if i % 2 == 0:
+                r = B.cdma_prefetch_direct(ctx, tickets[i], outs[i].data_ptr(), 0)
+            else:
+                r = B.cdma_prefetch(ctx, tickets[i], outs[i].data_ptr(), 0)
+            assert r == tensors[i].numel() * tensors[i].element_size(), B.status_string(r)
+            assert torch.equal(bits(outs[i]), bits(tensors[i]))
+        out = torch.zeros_like(tensors[0])
+        assert B.cdma_prefetch_direct(ctx, tk2, out.data_ptr(), 0) == out.numel() * out.element_size()
+        assert torch.equal(bits(out), bits(tensors[0]))
+        assert B.cdma_prefetch_direct(ctx, tk2, out.data_ptr(), 0) == -B.ERR_BAD_TICKET
+        # the worst-case reservation was given back: the pool takes the same set again
+        for t in tensors:
+            c, tk = B.cdma_offload_direct(ctx, t.data_ptr(), t.numel(), code, B.NCHW, 0)
+            assert c >= 0
+        assert B.cdma_ctx_synchronize(ctx) == 0
     finally:
         B.cdma_ctx_destroy(ctx)
