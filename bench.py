@@ -37,6 +37,7 @@ if ROOT not in sys.path:
 METRIC = "zvc_compress_decompress_uncompressed_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
+BASE_SEED_RELU = 170501626 + 6000
 NOMINAL_HBM_GBS = 8000.0
 
 # DRAM bytes per launch measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum),
@@ -707,6 +708,78 @@ def run_offload_set(args):
     B.cdma_ctx_destroy(ctx)
 
 
+def run_relu(args):
+    """ReLU + compression in one pass against ReLU (torch) followed by compression, on a
+    pre-activation tensor of the bench workload's shape whose ReLU has about the same density."""
+    import torch
+    from paper_1705_01626_b200 import binding as B
+    torch.cuda.set_device(0)
+    g = torch.Generator(device="cuda").manual_seed(BASE_SEED_RELU)
+    x = torch.empty(64, 64, 224, 224, device="cuda")
+    for b in range(64):
+        x[b] = torch.randn(64, 224, 224, generator=g, device="cuda") - 0.47
+    n = x.numel()
+    cap = B.cdma_zvc_max_compressed_bytes(n, B.F32)
+    entries = B.cdma_zvc_table_entries(n)
+    ws_bytes = B.cdma_zvc_workspace_bytes(n, B.F32)
+    payload = torch.empty(cap, dtype=torch.uint8, device="cuda")
+    payload2 = torch.empty(cap, dtype=torch.uint8, device="cuda")
+    table = torch.empty(entries, dtype=torch.int64, device="cuda")
+    table2 = torch.empty(entries, dtype=torch.int64, device="cuda")
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    y = torch.empty_like(x)
+    y2 = torch.empty_like(x)
+    res = torch.zeros(2, dtype=torch.int64).pin_memory()
+    sh = torch.cuda.current_stream().cuda_stream
+
+    def separate():
+        torch.clamp_min(x, 0.0, out=y)
+        B.cdma_zvc_compress_async(y.data_ptr(), n, B.F32, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
+                                  ws.data_ptr(), ws_bytes, sh, res.data_ptr())
+
+    def fused(with_dense):
+        B.cdma_zvc_relu_compress_async(x.data_ptr(), n, B.F32, B.NCHW, y2.data_ptr() if with_dense else 0,
+                                       payload2.data_ptr(), cap, table2.data_ptr(), ws.data_ptr(), ws_bytes, sh,
+                                       res.data_ptr())
+
+    separate()
+    torch.cuda.synchronize()
+    c = int(res[0])
+    fused(True)
+    torch.cuda.synchronize()
+    if int(res[0]) != c or not torch.equal(payload[:c], payload2[:c]) or not torch.equal(table, table2) \
+            or not torch.equal(y.view(torch.int32), y2.view(torch.int32)):
+        raise SystemExit("fused ReLU+compress differs from ReLU then compress")
+
+    def timed(fn, iters=30):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters
+
+    t_sep = timed(separate)
+    t_fd = timed(lambda: fused(True))
+    t_f = timed(lambda: fused(False))
+    dense = n * 4
+    peak, kind = measured_peak()
+    print(json.dumps({
+        "workload": "relu: fp32 64x64x224x224 pre-activations N(-0.47,1), ReLU density %.3f" % ((c - 4 * (n // 32)) / 4 / n),
+        "dense_bytes": dense, "compressed_bytes": c,
+        "relu_then_compress_ms": t_sep, "fused_with_dense_output_ms": t_fd, "fused_payload_only_ms": t_f,
+        "speedup_fused_with_dense": t_sep / t_fd, "speedup_payload_only": t_sep / t_f,
+        "algorithmic_bytes": {"relu_then_compress": 3 * dense + c, "fused_with_dense": 2 * dense + c,
+                              "fused_payload_only": dense + c},
+        "frac_of_" + kind: {"relu_then_compress": (3 * dense + c) / t_sep / 1e6 / peak,
+                            "fused_with_dense": (2 * dense + c) / t_fd / 1e6 / peak,
+                            "fused_payload_only": (dense + c) / t_f / 1e6 / peak}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -726,6 +799,8 @@ def main():
         run_offload_set(args)
     elif args.workload == "config4":
         run_sweep(args)
+    elif args.workload == "relu":
+        run_relu(args)
     else:
         run_cdma(args)
 

@@ -137,6 +137,32 @@ int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout
                             void* cuda_stream, uint64_t* h_result);
 
 /*
+ * Activation function and compression in one pass.  The sparsity this method
+ * exploits is produced by the ReLU layers (Section IV), and the paper leaves
+ * compressing "on the way into DRAM" as future work (Section IX): here the
+ * kernel reads the pre-activation tensor once, applies y = max(x, 0), and writes
+ * the compressed form of y -- and, when d_relu_out is not NULL, also the dense y
+ * for the next layer -- so y is never read back from memory to be compressed.
+ *
+ *   ReLU rule, on bit patterns: an element is kept unchanged when it is greater
+ *   than zero or a NaN of either sign (NaNs propagate, as in the usual framework
+ *   ReLU); every other value (negatives, -0.0, +0.0, -Inf) becomes +0.0.
+ *   d_relu_out   NULL, or n*s bytes, 16-byte aligned; may be d_src itself
+ *                (in-place activation) but must not overlap it otherwise, nor
+ *                the payload.
+ * Everything else, and the payload/table produced, is exactly that of
+ * cdma_zvc_compress applied to y.
+ */
+int64_t cdma_zvc_relu_compress(const void* d_src, uint64_t n, int dtype, int layout,
+                               void* d_relu_out, void* d_dst, uint64_t dst_capacity,
+                               uint64_t* d_table, void* d_workspace, uint64_t workspace_bytes,
+                               void* cuda_stream);
+int cdma_zvc_relu_compress_async(const void* d_src, uint64_t n, int dtype, int layout,
+                                 void* d_relu_out, void* d_dst, uint64_t dst_capacity,
+                                 uint64_t* d_table, void* d_workspace, uint64_t workspace_bytes,
+                                 void* cuda_stream, uint64_t* h_result);
+
+/*
  * The same compression for callers that cannot allocate device memory: code
  * inside a memory manager's eviction path (where an allocation could re-enter
  * the manager, or fail because the device is full -- which is when activations

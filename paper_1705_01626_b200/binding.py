@@ -53,6 +53,10 @@ _SIGNATURES = {
                                     c_void_p, c_uint64, c_void_p]),
     "cdma_zvc_compress_async": (c_int, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64, c_void_p,
                                         c_void_p, c_uint64, c_void_p, c_void_p]),
+    "cdma_zvc_relu_compress": (c_int64, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_void_p, c_uint64, c_void_p,
+                                         c_void_p, c_uint64, c_void_p]),
+    "cdma_zvc_relu_compress_async": (c_int, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_void_p, c_uint64, c_void_p,
+                                             c_void_p, c_uint64, c_void_p, c_void_p]),
     "cdma_zvc_compress_static_ws": (c_int64, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64, c_void_p,
                                               c_void_p]),
     "cdma_zvc_decompress": (c_int64, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p,
@@ -137,6 +141,21 @@ def cdma_zvc_compress_async(d_src, n, dtype, layout, d_dst, dst_capacity, d_tabl
     return int(lib().cdma_zvc_compress_async(_vp(d_src), n, dtype, layout, _vp(d_dst), dst_capacity,
                                              _vp(d_table), _vp(d_workspace), workspace_bytes,
                                              _vp(cuda_stream), _vp(h_result)))
+
+
+def cdma_zvc_relu_compress(d_src, n, dtype, layout, d_relu_out, d_dst, dst_capacity, d_table, d_workspace,
+                           workspace_bytes, cuda_stream=0) -> int:
+    """y = max(x, 0) and its compression in one pass; d_relu_out (may be 0) receives the dense y.
+    Returns the payload size C, or a negative status."""
+    return int(lib().cdma_zvc_relu_compress(_vp(d_src), n, dtype, layout, _vp(d_relu_out), _vp(d_dst), dst_capacity,
+                                            _vp(d_table), _vp(d_workspace), workspace_bytes, _vp(cuda_stream)))
+
+
+def cdma_zvc_relu_compress_async(d_src, n, dtype, layout, d_relu_out, d_dst, dst_capacity, d_table, d_workspace,
+                                 workspace_bytes, cuda_stream, h_result) -> int:
+    return int(lib().cdma_zvc_relu_compress_async(_vp(d_src), n, dtype, layout, _vp(d_relu_out), _vp(d_dst),
+                                                  dst_capacity, _vp(d_table), _vp(d_workspace), workspace_bytes,
+                                                  _vp(cuda_stream), _vp(h_result)))
 
 
 def cdma_zvc_compress_static_ws(d_src, n, dtype, layout, d_dst, dst_capacity, d_table, cuda_stream=0) -> int:

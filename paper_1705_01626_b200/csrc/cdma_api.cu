@@ -80,8 +80,9 @@ uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype) {
     return (bytes + 255) & ~255ull;
 }
 
-int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,
-                            uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
+// Shared body of the plain and the ReLU-fused compression calls.
+static int compress_enqueue(const void* d_src, uint64_t n, int dtype, int layout, bool relu, void* d_relu_out,
+                            void* d_dst, uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
                             uint64_t workspace_bytes, void* cuda_stream, uint64_t* h_result) {
     const int st = check_common(n, dtype, layout, d_src, d_dst, d_table, d_workspace, workspace_bytes);
     if (st != CDMA_OK) return st;
@@ -89,21 +90,57 @@ int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout
     if (h_result == nullptr) return CDMA_ERR_INVALID_ARG;
     const uint32_t s = cdma_dtype_size(dtype);
     if (overlaps(d_src, n * s, d_dst, dst_capacity)) return CDMA_ERR_INVALID_ARG;
+    if (relu && d_relu_out != nullptr) {
+        if (!aligned(d_relu_out, 16)) return CDMA_ERR_ALIGNMENT;
+        // writing the activation map over its own input is fine; over the payload it is not
+        if (overlaps(d_relu_out, n * s, d_dst, dst_capacity)) return CDMA_ERR_INVALID_ARG;
+        if (d_relu_out != d_src && overlaps(d_relu_out, n * s, d_src, n * s)) return CDMA_ERR_INVALID_ARG;
+    }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint64_t* ws = static_cast<uint64_t*>(d_workspace);
 
-    // ticket, result words and every tile descriptor start at zero
+    // result words and every tile descriptor start at zero
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * num_tiles_of(n), stream) != cudaSuccess)
         return CDMA_ERR_CUDA;
     if (n == 0) {
         if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return CDMA_ERR_CUDA;
-    } else if (launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, stream) !=
-               cudaSuccess) {
-        return CDMA_ERR_CUDA;
+    } else {
+        const uint32_t nan_above = (dtype == CDMA_F32) ? 0x7f800000u : (dtype == CDMA_F16 ? 0x7c00u : 0x7f80u);
+        const cudaError_t e =
+            relu ? launch_zvc_relu_compress(d_src, n, s, nan_above, d_relu_out, d_dst, dst_capacity, d_table, ws, stream)
+                 : launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, stream);
+        if (e != cudaSuccess) return CDMA_ERR_CUDA;
     }
     if (cudaMemcpyAsync(h_result, ws + kWsBytes, 16, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
         return CDMA_ERR_CUDA;
     return CDMA_OK;
+}
+
+int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,
+                            uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
+                            uint64_t workspace_bytes, void* cuda_stream, uint64_t* h_result) {
+    return compress_enqueue(d_src, n, dtype, layout, false, nullptr, d_dst, dst_capacity, d_table, d_workspace,
+                            workspace_bytes, cuda_stream, h_result);
+}
+
+int cdma_zvc_relu_compress_async(const void* d_src, uint64_t n, int dtype, int layout, void* d_relu_out,
+                                 void* d_dst, uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
+                                 uint64_t workspace_bytes, void* cuda_stream, uint64_t* h_result) {
+    return compress_enqueue(d_src, n, dtype, layout, true, d_relu_out, d_dst, dst_capacity, d_table, d_workspace,
+                            workspace_bytes, cuda_stream, h_result);
+}
+
+int64_t cdma_zvc_relu_compress(const void* d_src, uint64_t n, int dtype, int layout, void* d_relu_out,
+                               void* d_dst, uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
+                               uint64_t workspace_bytes, void* cuda_stream) {
+    uint64_t result[2] = {0, 0};
+    const int st = compress_enqueue(d_src, n, dtype, layout, true, d_relu_out, d_dst, dst_capacity, d_table,
+                                    d_workspace, workspace_bytes, cuda_stream, result);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (result[1] != 0) return -static_cast<int64_t>(result[1]);
+    return static_cast<int64_t>(result[0]);
 }
 
 int64_t cdma_zvc_compress(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,

@@ -73,6 +73,9 @@ __device__ __forceinline__ void report_status(uint64_t* ws, uint32_t code) {
 cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst,
                                 uint64_t cap, uint64_t* d_table, uint64_t* d_ws,
                                 cudaStream_t stream);
+cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
+                                     void* d_relu_out, void* d_dst, uint64_t cap, uint64_t* d_table,
+                                     uint64_t* d_ws, cudaStream_t stream);
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
                                   cudaStream_t stream);

@@ -91,11 +91,28 @@ __device__ __forceinline__ void load4(const uint16_t* p, uint32_t (&e)[4]) {
     e[0] = q.x & 0xffffu; e[1] = q.x >> 16; e[2] = q.y & 0xffffu; e[3] = q.y >> 16;
 }
 
-template <typename T>
+// ReLU on bit patterns, NaN-propagating: an element is kept when it is greater
+// than zero or a NaN (of either sign); everything else -- negatives, -0.0, +0.0,
+// -Inf -- becomes +0.  `nan_above` is the largest magnitude pattern that is not a
+// NaN (0x7f800000 for fp32, 0x7c00 for fp16, 0x7f80 for bf16).
+__device__ __forceinline__ uint32_t relu_bits32(uint32_t e) {
+    const bool keep = (static_cast<int32_t>(e) > 0) || ((e & 0x7fffffffu) > 0x7f800000u);
+    return keep ? e : 0u;
+}
+__device__ __forceinline__ uint32_t relu_bits16(uint32_t h, uint32_t nan_above) {
+    const bool keep = ((h & 0x8000u) == 0u && h != 0u) || ((h & 0x7fffu) > nan_above);
+    return keep ? h : 0u;
+}
+
+// When RELU is set the kernel compresses max(x, 0) instead of x (the activation
+// function whose output the paper offloads, Section IV) and, if relu_out is not
+// null, also writes the dense activation map for the next layer -- the input is
+// read once for both.
+template <typename T, bool RELU>
 __global__ void __launch_bounds__(kTileThreads, 3)
 zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
                     uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
-                    uint64_t num_chunks) {
+                    uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above) {
     constexpr uint32_t S = sizeof(T);
     constexpr uint32_t MU = 4 / S;                              // units of T per mask
     constexpr uint32_t kMaxChunkUnits = MU * kChunkWindows + kChunk;
@@ -130,6 +147,16 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
         const T* p = src + e0 + 4 * lane;
 #pragma unroll
         for (uint32_t g = 0; g < kGroups; ++g) load4(p + g * 128, e[g]);
+        if (RELU) {
+#pragma unroll
+            for (uint32_t g = 0; g < kGroups; ++g) {
+#pragma unroll
+                for (uint32_t k = 0; k < 4; ++k) e[g][k] = relu_bits32(e[g][k]);
+                if (relu_out != nullptr)
+                    *reinterpret_cast<uint4*>(relu_out + e0 + 4 * lane + g * 128) =
+                        make_uint4(e[g][0], e[g][1], e[g][2], e[g][3]);
+            }
+        }
     } else {
         const uint64_t left = (e0 < n) ? (n - e0) : 0;
         nwin = static_cast<uint32_t>((left + kWindow - 1) / kWindow);
@@ -139,6 +166,10 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
             for (uint32_t k = 0; k < 4; ++k) {
                 const uint64_t j = static_cast<uint64_t>(g) * 128 + 4 * lane + k;
                 e[g][k] = (j < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j)) : 0u;
+                if (RELU) {
+                    e[g][k] = relu_bits32(e[g][k]);
+                    if (relu_out != nullptr && j < left) relu_out[e0 + j] = static_cast<T>(e[g][k]);
+                }
             }
         }
     }
@@ -247,10 +278,12 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
 // kernel and the look-back runs at the same rate per byte.
 constexpr uint32_t kTileChunksU16 = 2 * kTileChunks;
 
+template <bool RELU>
 __global__ void __launch_bounds__(kTileThreads, 3)
 zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst,
                         uint64_t cap, uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
-                        uint32_t num_tiles, uint64_t num_chunks) {
+                        uint32_t num_tiles, uint64_t num_chunks, uint16_t* __restrict__ relu_out,
+                        uint32_t nan_above) {
     using T = uint16_t;
     constexpr uint32_t S = 2, MU = 2;
     constexpr uint32_t kMaxChunkUnits = MU * kChunkWindows + kChunk;
@@ -283,6 +316,15 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
             for (uint32_t g = 0; g < kGroups; ++g) {
                 const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p + g * 256));
                 w[c][g][0] = q.x; w[c][g][1] = q.y; w[c][g][2] = q.z; w[c][g][3] = q.w;
+                if (RELU) {
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k)
+                        w[c][g][k] = relu_bits16(w[c][g][k] & 0xffffu, nan_above) |
+                                     (relu_bits16(w[c][g][k] >> 16, nan_above) << 16);
+                    if (relu_out != nullptr)
+                        *reinterpret_cast<uint4*>(relu_out + e0 + 8 * lane + g * 256) =
+                            make_uint4(w[c][g][0], w[c][g][1], w[c][g][2], w[c][g][3]);
+                }
             }
         } else {
             const uint64_t left = (e0 < n) ? (n - e0) : 0;
@@ -292,8 +334,14 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
 #pragma unroll
                 for (uint32_t k = 0; k < 4; ++k) {
                     const uint64_t j = static_cast<uint64_t>(g) * 256 + 8 * lane + 2 * k;
-                    const uint32_t lo = (j < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j)) : 0u;
-                    const uint32_t hi = (j + 1 < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j + 1)) : 0u;
+                    uint32_t lo = (j < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j)) : 0u;
+                    uint32_t hi = (j + 1 < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j + 1)) : 0u;
+                    if (RELU) {
+                        lo = relu_bits16(lo, nan_above);
+                        hi = relu_bits16(hi, nan_above);
+                        if (relu_out != nullptr && j < left) relu_out[e0 + j] = static_cast<T>(lo);
+                        if (relu_out != nullptr && j + 1 < left) relu_out[e0 + j + 1] = static_cast<T>(hi);
+                    }
                     w[c][g][k] = lo | (hi << 16);
                 }
             }
@@ -415,7 +463,8 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
 
 template <typename T, uint32_t TILE_CHUNKS, typename Kernel>
 cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_dst, uint64_t cap,
-                         uint64_t* d_table, uint64_t* d_ws, cudaStream_t stream) {
+                         uint64_t* d_table, uint64_t* d_ws, void* d_relu_out, uint32_t nan_above,
+                         cudaStream_t stream) {
     constexpr uint32_t kSmem = TILE_CHUNKS * (4 * kChunkWindows + sizeof(T) * kChunk);
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
@@ -423,7 +472,7 @@ cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_d
     const uint64_t tiles = (chunks + TILE_CHUNKS - 1) / TILE_CHUNKS;   // never more than num_tiles_of(n)
     kernel<<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
         static_cast<const T*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
-        static_cast<uint32_t>(tiles), chunks);
+        static_cast<uint32_t>(tiles), chunks, static_cast<T*>(d_relu_out), nan_above);
     return cudaGetLastError();
 }
 
@@ -435,8 +484,24 @@ cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_siz
     if (num_tiles_of(n) == 0) return cudaSuccess;
     const cudaError_t e =
         (elem_size == 4)
-            ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t>, d_src, n, d_dst, cap, d_table, d_ws, stream)
-            : launch_typed<uint16_t, kTileChunksU16>(zvc_compress_kernel_u16, d_src, n, d_dst, cap, d_table, d_ws, stream);
+            ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t, false>, d_src, n, d_dst, cap,
+                                                  d_table, d_ws, nullptr, 0, stream)
+            : launch_typed<uint16_t, kTileChunksU16>(zvc_compress_kernel_u16<false>, d_src, n, d_dst, cap,
+                                                     d_table, d_ws, nullptr, 0, stream);
+    count_kernel_launch();
+    return e;
+}
+
+cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
+                                     void* d_relu_out, void* d_dst, uint64_t cap, uint64_t* d_table,
+                                     uint64_t* d_ws, cudaStream_t stream) {
+    if (num_tiles_of(n) == 0) return cudaSuccess;
+    const cudaError_t e =
+        (elem_size == 4)
+            ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t, true>, d_src, n, d_dst, cap,
+                                                  d_table, d_ws, d_relu_out, nan_above, stream)
+            : launch_typed<uint16_t, kTileChunksU16>(zvc_compress_kernel_u16<true>, d_src, n, d_dst, cap,
+                                                     d_table, d_ws, d_relu_out, nan_above, stream);
     count_kernel_launch();
     return e;
 }
