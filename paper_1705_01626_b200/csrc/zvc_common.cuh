@@ -16,7 +16,14 @@ constexpr uint32_t kChunkWindows = 32;
 constexpr uint32_t kChunk = kWindow * kChunkWindows;   // 1024 elements
 
 // Compression tiling: one CTA = one tile = kTileChunks chunks, one warp per chunk.
-constexpr uint32_t kTileChunks = 12;
+#ifndef CDMA_TILE_CHUNKS
+#define CDMA_TILE_CHUNKS 12
+#endif
+#ifndef CDMA_MIN_CTAS
+#define CDMA_MIN_CTAS 3
+#endif
+constexpr uint32_t kTileChunks = CDMA_TILE_CHUNKS;
+constexpr uint32_t kMinCtasPerSm = CDMA_MIN_CTAS;
 constexpr uint32_t kTileThreads = 32 * kTileChunks;
 
 // Workspace layout, in uint64 words.

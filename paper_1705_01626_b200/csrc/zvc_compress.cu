@@ -91,6 +91,24 @@ __device__ __forceinline__ void load4(const uint16_t* p, uint32_t (&e)[4]) {
     e[0] = q.x & 0xffffu; e[1] = q.x >> 16; e[2] = q.y & 0xffffu; e[3] = q.y >> 16;
 }
 
+// Tiles follow the block index and blocks are dispatched in that order, so the
+// tile `kPrefetchAhead` places further on will be picked up by a CTA that starts
+// about one CTA lifetime from now (3 CTAs x 148 SMs are resident at a time).
+// Asking L2 for it now turns that CTA's DRAM-latency load phase into L2 hits;
+// every line is still fetched from DRAM exactly once.
+#ifndef CDMA_PREFETCH_AHEAD
+#define CDMA_PREFETCH_AHEAD 444
+#endif
+constexpr uint32_t kPrefetchAhead = CDMA_PREFETCH_AHEAD;
+constexpr uint32_t kTileBytes = kTileChunks * kChunk * 4;      // 48 KB for either element width
+
+__device__ __forceinline__ void prefetch_future_tile(const void* src, uint64_t total_bytes, uint32_t tile) {
+    if (kPrefetchAhead == 0) return;
+    const uint64_t off = (static_cast<uint64_t>(tile) + kPrefetchAhead) * kTileBytes + 128ull * threadIdx.x;
+    if (off + 128 <= total_bytes)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const uint8_t*>(src) + off));
+}
+
 // ReLU on bit patterns, NaN-propagating: an element is kept when it is greater
 // than zero or a NaN (of either sign); everything else -- negatives, -0.0, +0.0,
 // -Inf -- becomes +0.  `nan_above` is the largest magnitude pattern that is not a
@@ -109,7 +127,7 @@ __device__ __forceinline__ uint32_t relu_bits16(uint32_t h, uint32_t nan_above) 
 // null, also writes the dense activation map for the next layer -- the input is
 // read once for both.
 template <typename T, bool RELU>
-__global__ void __launch_bounds__(kTileThreads, 3)
+__global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
 zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
                     uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
                     uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above) {
@@ -136,6 +154,7 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     // ever not hold, the bounded wait below turns it into CDMA_ERR_TIMEOUT.
     const uint32_t tile = blockIdx.x;
     if (tile >= num_tiles) return;
+    prefetch_future_tile(src, n * S, tile);
 
     // ---- load the warp's chunk: 8 vector loads per lane, all in flight ------
     const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunks + warp;
@@ -279,7 +298,7 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
 constexpr uint32_t kTileChunksU16 = 2 * kTileChunks;
 
 template <bool RELU>
-__global__ void __launch_bounds__(kTileThreads, 3)
+__global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
 zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst,
                         uint64_t cap, uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
                         uint32_t num_tiles, uint64_t num_chunks, uint16_t* __restrict__ relu_out,
@@ -302,6 +321,7 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
     uint64_t* desc = ws + kWsDescriptors;
     const uint32_t tile = blockIdx.x;     // block-index order, as in the 4-byte kernel
     if (tile >= num_tiles) return;
+    prefetch_future_tile(src, n * S, tile);
 
     // ---- load the warp's two chunks ------------------------------------------
     uint32_t nwin[2];
