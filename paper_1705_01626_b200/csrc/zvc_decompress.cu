@@ -21,6 +21,10 @@ namespace {
 
 constexpr uint32_t kDecWarps = 8;
 constexpr uint32_t kDecThreads = 32 * kDecWarps;
+#ifndef CDMA_DEC_PREFETCH_CTAS
+#define CDMA_DEC_PREFETCH_CTAS 888
+#endif
+constexpr uint32_t kPrefetchAheadCtas = CDMA_DEC_PREFETCH_CTAS;   // 6 CTAs x 148 SMs resident at a time
 
 __device__ __forceinline__ void store4(uint32_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     __stcs(reinterpret_cast<uint4*>(p), make_uint4(a, b, c, d));
@@ -29,7 +33,7 @@ __device__ __forceinline__ void store4(uint16_t* p, uint32_t a, uint32_t b, uint
     __stcs(reinterpret_cast<uint2*>(p), make_uint2(a | (b << 16), c | (d << 16)));
 }
 
-template <typename T>
+template <typename T, bool PREFETCH>
 __global__ void __launch_bounds__(kDecThreads)
 zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
                       const uint64_t* __restrict__ table, uint64_t n, T* __restrict__ dst,
@@ -91,6 +95,23 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
             q = make_uint4(wds[0], wds[1], wds[2], wds[3]);
         }
         *reinterpret_cast<uint4*>(buf + (a - a0)) = q;
+    }
+    // Blocks are dispatched in index order, so the chunk `kPrefetchAheadCtas` blocks
+    // further on will be expanded by a warp that starts about one CTA lifetime from
+    // now: ask L2 for its table entries (by reading them) and its payload bytes now.
+    // Nothing depends on this and every line still comes from DRAM exactly once.
+    // Worth its instructions only where the payload is a sizeable part of the traffic:
+    // the launcher picks this variant by the payload-to-dense ratio.
+    if (PREFETCH && kPrefetchAheadCtas != 0) {
+        const uint64_t cf = chunk + static_cast<uint64_t>(kPrefetchAheadCtas) * kDecWarps;
+        if (cf < num_chunks) {
+            const uint64_t flo = __ldg(table + cf);
+            const uint64_t fhi = __ldg(table + cf + 1);
+            if (flo <= fhi && fhi <= src_bytes && fhi - flo <= kMaxChunkBytes) {
+                for (uint64_t a = (flo & ~127ull) + 128ull * lane; a < fhi; a += 128ull * 32)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src + a));
+            }
+        }
     }
     __syncwarp();
 
@@ -162,11 +183,13 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
     if (chunks == 0) return cudaSuccess;
     const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
     if (elem_size == 4) {
-        zvc_decompress_kernel<uint32_t><<<grid, kDecThreads, 0, stream>>>(
-            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint32_t*>(d_dst),
-            d_ws, chunks);
+        // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
+        const bool prefetch = src_bytes >= (n * 4) / 5;
+        auto kernel = prefetch ? zvc_decompress_kernel<uint32_t, true> : zvc_decompress_kernel<uint32_t, false>;
+        kernel<<<grid, kDecThreads, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes, d_table, n,
+                                                 static_cast<uint32_t*>(d_dst), d_ws, chunks);
     } else {
-        zvc_decompress_kernel<uint16_t><<<grid, kDecThreads, 0, stream>>>(
+        zvc_decompress_kernel<uint16_t, false><<<grid, kDecThreads, 0, stream>>>(
             static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint16_t*>(d_dst),
             d_ws, chunks);
     }
