@@ -312,6 +312,13 @@ int64_t cdma_zvc_decompress_host(cdma_ctx* ctx, const void* h_src, uint64_t src_
                                  const uint64_t* h_table, uint64_t n, int dtype, int layout,
                                  void* h_dst);
 
+/* Measurement hook: the next codec kernel this thread launches (compress or
+ * decompress, through any entry point) is bracketed by cudaEventRecord of the
+ * two given cudaEvent_t handles on the launch stream, around the kernel alone
+ * (not the workspace reset or the result copy of the call).  One-shot: the pair
+ * is forgotten after that launch.  Pass NULLs to cancel. */
+void cdma_time_next_kernel(void* start_event, void* stop_event);
+
 /* Number of kernel launches this library has issued in this process (codec
  * kernels only; memsets and copies are not counted). */
 uint64_t cdma_kernel_launch_count(void);

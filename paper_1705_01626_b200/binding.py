@@ -77,6 +77,7 @@ _SIGNATURES = {
                                          c_void_p]),
     "cdma_zvc_decompress_host": (c_int64, [c_void_p, c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int,
                                            c_void_p]),
+    "cdma_time_next_kernel": (None, [c_void_p, c_void_p]),
     "cdma_kernel_launch_count": (c_uint64, []),
 }
 
@@ -247,6 +248,12 @@ def cdma_zvc_compress_host(ctx, h_src, n, dtype, layout, h_dst, dst_capacity, h_
 def cdma_zvc_decompress_host(ctx, h_src, src_bytes, h_table, n, dtype, layout, h_dst) -> int:
     return int(lib().cdma_zvc_decompress_host(ctx, _vp(h_src), src_bytes, _vp(h_table), n, dtype, layout,
                                               _vp(h_dst)))
+
+
+def cdma_time_next_kernel(start_event, stop_event) -> None:
+    """Bracket the next codec kernel launch of this thread with the two cudaEvent_t handles
+    (e.g. ``torch.cuda.Event(enable_timing=True).cuda_event`` after a first ``record()``)."""
+    lib().cdma_time_next_kernel(_vp(start_event), _vp(stop_event))
 
 
 def cdma_kernel_launch_count() -> int:

@@ -10,6 +10,18 @@ namespace cdma {
 static std::atomic<uint64_t> g_kernel_launches{0};
 void count_kernel_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
 
+// One-shot pair of events that the next codec kernel launch of this thread is bracketed with.
+static thread_local cudaEvent_t t_time_start = nullptr;
+static thread_local cudaEvent_t t_time_stop = nullptr;
+void timing_before_launch(cudaStream_t stream) {
+    if (t_time_start != nullptr) cudaEventRecord(t_time_start, stream);
+}
+void timing_after_launch(cudaStream_t stream) {
+    if (t_time_stop != nullptr) cudaEventRecord(t_time_stop, stream);
+    t_time_start = nullptr;
+    t_time_stop = nullptr;
+}
+
 static inline bool aligned(const void* p, uintptr_t a) {
     return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0;
 }
@@ -192,6 +204,11 @@ int64_t cdma_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_
         return -static_cast<int64_t>(CDMA_ERR_CUDA);
     if (result[1] != 0) return -static_cast<int64_t>(result[1]);
     return static_cast<int64_t>(n) * cdma_dtype_size(dtype);
+}
+
+void cdma_time_next_kernel(void* start_event, void* stop_event) {
+    t_time_start = static_cast<cudaEvent_t>(start_event);
+    t_time_stop = static_cast<cudaEvent_t>(stop_event);
 }
 
 uint64_t cdma_kernel_launch_count(void) { return g_kernel_launches.load(std::memory_order_relaxed); }

@@ -87,5 +87,7 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
                                   cudaStream_t stream);
 void count_kernel_launch();
+void timing_before_launch(cudaStream_t stream);   // measurement hook, see cdma_time_next_kernel
+void timing_after_launch(cudaStream_t stream);
 
 }  // namespace cdma

@@ -490,9 +490,11 @@ cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_d
     if (e != cudaSuccess) return e;
     const uint64_t chunks = num_chunks_of(n);
     const uint64_t tiles = (chunks + TILE_CHUNKS - 1) / TILE_CHUNKS;   // never more than num_tiles_of(n)
+    timing_before_launch(stream);
     kernel<<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
         static_cast<const T*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
         static_cast<uint32_t>(tiles), chunks, static_cast<T*>(d_relu_out), nan_above);
+    timing_after_launch(stream);
     return cudaGetLastError();
 }
 

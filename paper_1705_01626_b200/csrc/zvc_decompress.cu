@@ -182,6 +182,7 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
     const uint64_t chunks = num_chunks_of(n);
     if (chunks == 0) return cudaSuccess;
     const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
+    timing_before_launch(stream);
     if (elem_size == 4) {
         // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
         const bool prefetch = src_bytes >= (n * 4) / 5;
@@ -193,6 +194,7 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
             static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint16_t*>(d_dst),
             d_ws, chunks);
     }
+    timing_after_launch(stream);
     count_kernel_launch();
     return cudaGetLastError();
 }
