@@ -122,6 +122,41 @@ __device__ __forceinline__ uint32_t relu_bits16(uint32_t h, uint32_t nan_above) 
     return keep ? h : 0u;
 }
 
+// Records of one chunk into shared memory, one window per step: the ballot of
+// "my element is non-zero" IS the window's mask (compare stage), the pop-count of
+// the mask bits below a lane is the slot of its value (prefix-sum and shift
+// stages), lane 0 appends the mask word itself.  Returns the units written.
+// (The two stores are predicated instructions, not branches: a divergent branch
+// in front of every ballot would cost a reconvergence point per window.)
+__device__ __forceinline__ void sts_if(uint32_t saddr, uint32_t v, bool pred) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %1;\n\t}"
+                 ::"r"(saddr), "r"(v), "r"(static_cast<uint32_t>(pred)) : "memory");
+}
+
+template <bool FULL>
+__device__ __forceinline__ uint32_t assemble_chunk(uint32_t* st, const uint32_t (&e)[kChunkWindows], uint32_t nwin,
+                                                   uint32_t lane, uint32_t lt) {
+    const uint32_t base = static_cast<uint32_t>(__cvta_generic_to_shared(st));
+    const bool first = lane == 0;
+    uint32_t pos = 0;                                           // bytes written so far
+#pragma unroll
+    for (uint32_t w = 0; w < kChunkWindows; ++w) {
+        if (!FULL && w >= nwin) break;
+        const bool nz = e[w] != 0u;
+        const uint32_t m = __ballot_sync(0xffffffffu, nz);
+        sts_if(base + pos, m, first);
+        sts_if(base + pos + 4 + 4 * __popc(m & lt), e[w], nz);
+        pos += 4 + 4 * __popc(m);
+    }
+    return pos / 4;
+}
+
+// 4-byte elements.  A lane holds one element of each of the chunk's 32 windows
+// (warp loads are 128 contiguous bytes), so a window's mask is one warp ballot.
+// The tile's records are staged contiguously in shared memory -- each chunk at
+// the offset the count step gave it -- and the whole CTA then copies them out
+// with stores that each cover one aligned 128-byte line.
+//
 // When RELU is set the kernel compresses max(x, 0) instead of x (the activation
 // function whose output the paper offloads, Section IV) and, if relu_out is not
 // null, also writes the dense activation map for the next layer -- the input is
@@ -131,21 +166,17 @@ __global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
 zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
                     uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
                     uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above) {
-    constexpr uint32_t S = sizeof(T);
-    constexpr uint32_t MU = 4 / S;                              // units of T per mask
-    constexpr uint32_t kMaxChunkUnits = MU * kChunkWindows + kChunk;
-    constexpr uint32_t kGroups = kChunk / 128;                  // 128 elements per warp load
+    static_assert(sizeof(T) == 4, "2-byte elements have a kernel of their own");
+    constexpr uint32_t S = 4;
     extern __shared__ __align__(16) uint8_t smem_raw[];
-    T (*stage)[kMaxChunkUnits] = reinterpret_cast<T (*)[kMaxChunkUnits]>(smem_raw);
+    uint32_t* s_tile = reinterpret_cast<uint32_t*>(smem_raw);   // up to kTileChunks * 1056 units
     __shared__ uint32_t s_chunk_units[kTileChunks];
-    __shared__ uint32_t s_chunk_off[kTileChunks];
     __shared__ uint64_t s_base;
     __shared__ uint32_t s_failed;
 
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
-    const uint32_t sub = lane & 7u;       // position of this lane's nibble in its window
-    const uint32_t wj = lane >> 3;        // which of the 4 windows of a group
+    const uint32_t lt = lanemask_lt();
     uint64_t* desc = ws + kWsDescriptors;
 
     // Tile = block index.  Thread blocks are dispatched in increasing index order,
@@ -156,106 +187,59 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     if (tile >= num_tiles) return;
     prefetch_future_tile(src, n * S, tile);
 
-    // ---- load the warp's chunk: 8 vector loads per lane, all in flight ------
+    // ---- load the warp's chunk: 32 loads per lane, all in flight --------------
     const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunks + warp;
     const uint64_t e0 = chunk * kChunk;
     uint32_t nwin;   // windows this chunk really has
-    uint32_t e[kGroups][4];
+    uint32_t e[kChunkWindows];
     if (e0 + kChunk <= n) {
         nwin = kChunkWindows;
-        const T* p = src + e0 + 4 * lane;
+        const T* p = src + e0 + lane;
 #pragma unroll
-        for (uint32_t g = 0; g < kGroups; ++g) load4(p + g * 128, e[g]);
+        for (uint32_t w = 0; w < kChunkWindows; ++w) e[w] = __ldcs(p + w * kWindow);
         if (RELU) {
 #pragma unroll
-            for (uint32_t g = 0; g < kGroups; ++g) {
-#pragma unroll
-                for (uint32_t k = 0; k < 4; ++k) e[g][k] = relu_bits32(e[g][k]);
-                if (relu_out != nullptr)
-                    *reinterpret_cast<uint4*>(relu_out + e0 + 4 * lane + g * 128) =
-                        make_uint4(e[g][0], e[g][1], e[g][2], e[g][3]);
+            for (uint32_t w = 0; w < kChunkWindows; ++w) {
+                e[w] = relu_bits32(e[w]);
+                if (relu_out != nullptr) relu_out[e0 + lane + w * kWindow] = e[w];
             }
         }
     } else {
         const uint64_t left = (e0 < n) ? (n - e0) : 0;
         nwin = static_cast<uint32_t>((left + kWindow - 1) / kWindow);
 #pragma unroll
-        for (uint32_t g = 0; g < kGroups; ++g) {
-#pragma unroll
-            for (uint32_t k = 0; k < 4; ++k) {
-                const uint64_t j = static_cast<uint64_t>(g) * 128 + 4 * lane + k;
-                e[g][k] = (j < left) ? static_cast<uint32_t>(__ldcs(src + e0 + j)) : 0u;
-                if (RELU) {
-                    e[g][k] = relu_bits32(e[g][k]);
-                    if (relu_out != nullptr && j < left) relu_out[e0 + j] = static_cast<T>(e[g][k]);
-                }
+        for (uint32_t w = 0; w < kChunkWindows; ++w) {
+            const uint64_t j = static_cast<uint64_t>(w) * kWindow + lane;
+            e[w] = (j < left) ? __ldcs(src + e0 + j) : 0u;
+            if (RELU) {
+                e[w] = relu_bits32(e[w]);
+                if (relu_out != nullptr && j < left) relu_out[e0 + j] = e[w];
             }
         }
     }
 
-    // ---- 1. count: 4 "non-zero" bits per group, 8 groups packed in one word --
-    uint32_t nibs = 0;
+    // ---- 1. count: the tile's size needs only the number of non-zeros ---------
+    uint32_t mine = 0;
 #pragma unroll
-    for (uint32_t g = 0; g < kGroups; ++g) {
-        const uint32_t nib = (e[g][0] != 0u ? 1u : 0u) | (e[g][1] != 0u ? 2u : 0u) |
-                             (e[g][2] != 0u ? 4u : 0u) | (e[g][3] != 0u ? 8u : 0u);
-        nibs |= nib << (4 * g);
-    }
-    const uint32_t units = MU * nwin + __reduce_add_sync(0xffffffffu, __popc(nibs));
+    for (uint32_t w = 0; w < kChunkWindows; ++w) mine += (e[w] != 0u) ? 1u : 0u;
+    const uint32_t units = nwin + __reduce_add_sync(0xffffffffu, mine);
     if (lane == 0) s_chunk_units[warp] = units;
     __syncthreads();
+    // every warp sums the chunks in front of its own; warp 0 also needs the total
+    const uint32_t cu = (lane < kTileChunks) ? s_chunk_units[lane] : 0u;
+    const uint32_t chunk_off = __reduce_add_sync(0xffffffffu, lane < warp ? cu : 0u);
     uint64_t tile_bytes = 0;
     if (warp == 0) {
-        const uint32_t cu = (lane < kTileChunks) ? s_chunk_units[lane] : 0u;
-        uint32_t ci = cu;
-#pragma unroll
-        for (int o = 1; o < static_cast<int>(kTileChunks); o <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xffffffffu, ci, o);
-            if (lane >= static_cast<uint32_t>(o)) ci += t;
-        }
-        if (lane < kTileChunks) s_chunk_off[lane] = ci - cu;
-        tile_bytes = static_cast<uint64_t>(__shfl_sync(0xffffffffu, ci, kTileChunks - 1)) * S;
+        tile_bytes = static_cast<uint64_t>(__reduce_add_sync(0xffffffffu, cu)) * S;
         // the tile's size is public before any record is assembled
         if (lane == 0)
             st_relaxed_u64(desc + tile, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
     }
 
-    // ---- 2. assemble the chunk's records in shared memory --------------------
-    T* st = stage[warp];
-    uint32_t run = 0;                     // units of T emitted so far by this chunk
-    const uint32_t below = (1u << (4 * sub)) - 1u;
-#pragma unroll
-    for (uint32_t g = 0; g < kGroups; ++g) {
-        const uint32_t nib = (nibs >> (4 * g)) & 15u;
-        uint32_t m = nib << (4 * sub);
-        m |= __shfl_xor_sync(0xffffffffu, m, 1);
-        m |= __shfl_xor_sync(0xffffffffu, m, 2);
-        m |= __shfl_xor_sync(0xffffffffu, m, 4);               // the window's 32-bit mask
-        const bool live = (g * 4 + wj) < nwin;
-        const uint32_t rec = live ? (MU + __popc(m)) : 0u;     // record length, same in 8 lanes
-        uint32_t incl = rec;
-        uint32_t t = __shfl_up_sync(0xffffffffu, incl, 8);
-        if (lane >= 8) incl += t;
-        t = __shfl_up_sync(0xffffffffu, incl, 16);
-        if (lane >= 16) incl += t;                             // records of windows <= wj
-        const uint32_t pos = run + incl - rec;                 // where this window's record starts
-        run += __shfl_sync(0xffffffffu, incl, 31);
-        if (live) {
-            if (sub == 0) {
-                if (S == 4) {
-                    st[pos] = static_cast<T>(m);
-                } else {
-                    st[pos] = static_cast<T>(m & 0xffffu);
-                    st[pos + 1] = static_cast<T>(m >> 16);
-                }
-            }
-            uint32_t q = pos + MU + __popc(m & below);
-            if (nib & 1u) st[q++] = static_cast<T>(e[g][0]);
-            if (nib & 2u) st[q++] = static_cast<T>(e[g][1]);
-            if (nib & 4u) st[q++] = static_cast<T>(e[g][2]);
-            if (nib & 8u) st[q] = static_cast<T>(e[g][3]);
-        }
-    }
+    // ---- 2. assemble the chunk's records at its place in the staged tile ------
+    uint32_t* st = s_tile + chunk_off;
+    if (nwin == kChunkWindows) assemble_chunk<true>(st, e, nwin, lane, lt);
+    else assemble_chunk<false>(st, e, nwin, lane, lt);
 
     // ---- 3. the tile's place in the stream ------------------------------------
     if (warp == 0) {
@@ -281,14 +265,21 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     __syncthreads();
     if (s_failed) return;
 
-    // ---- 4. each warp writes its chunk's bytes to their place, below cap ------
-    const uint64_t first_unit = s_base / S + s_chunk_off[warp];
-    if (lane == 0 && chunk < num_chunks) table[chunk] = first_unit * S;
+    // ---- 4. the CTA writes the tile's bytes to their place, below cap ---------
+    const uint64_t first_unit = s_base / S;
+    if (lane == 0 && chunk < num_chunks) table[chunk] = (first_unit + chunk_off) * S;
+    uint32_t tile_units = 0;                                    // same sum in every warp
+#pragma unroll
+    for (uint32_t c = 0; c < kTileChunks; ++c) tile_units += s_chunk_units[c];
     const uint64_t cap_units = cap / S;
-    T* out = reinterpret_cast<T*>(dst) + first_unit;
     const uint32_t room = (first_unit >= cap_units) ? 0u
-                        : (cap_units - first_unit < run ? static_cast<uint32_t>(cap_units - first_unit) : run);
-    for (uint32_t i = lane; i < room; i += 32) out[i] = st[i];
+                        : (cap_units - first_unit < tile_units ? static_cast<uint32_t>(cap_units - first_unit)
+                                                               : tile_units);
+    uint32_t* out = reinterpret_cast<uint32_t*>(dst) + first_unit;
+    // units in front of the first 128-byte line boundary of the destination
+    const uint32_t head = min(room, (32u - static_cast<uint32_t>(first_unit & 31u)) & 31u);
+    if (threadIdx.x < head) out[threadIdx.x] = s_tile[threadIdx.x];
+    for (uint32_t u = head + threadIdx.x; u < room; u += kTileThreads) out[u] = s_tile[u];
 }
 
 // 2-byte elements: the same four steps with 8 consecutive elements per lane (one
