@@ -126,29 +126,48 @@ __device__ __forceinline__ uint32_t relu_bits16(uint32_t h, uint32_t nan_above) 
 // "my element is non-zero" IS the window's mask (compare stage), the pop-count of
 // the mask bits below a lane is the slot of its value (prefix-sum and shift
 // stages), lane 0 appends the mask word itself.  Returns the units written.
-// (The two stores are predicated instructions, not branches: a divergent branch
-// in front of every ballot would cost a reconvergence point per window.)
-__device__ __forceinline__ void sts_if(uint32_t saddr, uint32_t v, bool pred) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %1;\n\t}"
-                 ::"r"(saddr), "r"(v), "r"(static_cast<uint32_t>(pred)) : "memory");
+// One window of a chunk, written as one block of PTX so that it stays at nine
+// instructions (the kernel is bound by instruction issue, not by DRAM, once the
+// loads are prefetched): compare, ballot, mask store (all lanes, same address,
+// same value), rank = popc(mask & lanes below), predicated value store, record
+// length.  `a` is the shared-memory byte address of the window's record minus
+// 4*W, so that the 4 bytes of every mask word in front fold into the immediate
+// offsets; no branch, hence no reconvergence point in front of the ballot.
+template <uint32_t W>
+__device__ __forceinline__ void assemble_window(uint32_t& a, uint32_t e, uint32_t lt) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b32 m, t, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "vote.sync.ballot.b32 m, p, 0xffffffff;\n\t"
+        "st.shared.u32 [%0+%3], m;\n\t"
+        "and.b32 t, m, %2;\n\t"
+        "popc.b32 t, t;\n\t"
+        "mad.lo.u32 q, t, 4, %0;\n\t"
+        "@p st.shared.u32 [q+%4], %1;\n\t"
+        "popc.b32 t, m;\n\t"
+        "mad.lo.u32 %0, t, 4, %0;\n\t"
+        "}"
+        : "+r"(a)
+        : "r"(e), "r"(lt), "n"(4 * W), "n"(4 * W + 4)
+        : "memory");
 }
 
-template <bool FULL>
-__device__ __forceinline__ uint32_t assemble_chunk(uint32_t* st, const uint32_t (&e)[kChunkWindows], uint32_t nwin,
-                                                   uint32_t lane, uint32_t lt) {
-    const uint32_t base = static_cast<uint32_t>(__cvta_generic_to_shared(st));
-    const bool first = lane == 0;
-    uint32_t pos = 0;                                           // bytes written so far
-#pragma unroll
-    for (uint32_t w = 0; w < kChunkWindows; ++w) {
-        if (!FULL && w >= nwin) break;
-        const bool nz = e[w] != 0u;
-        const uint32_t m = __ballot_sync(0xffffffffu, nz);
-        sts_if(base + pos, m, first);
-        sts_if(base + pos + 4 + 4 * __popc(m & lt), e[w], nz);
-        pos += 4 + 4 * __popc(m);
+template <uint32_t W>
+__device__ __forceinline__ void assemble_windows(uint32_t& a, const uint32_t (&e)[kChunkWindows], uint32_t nwin,
+                                                 uint32_t lt) {
+    if constexpr (W < kChunkWindows) {
+        if (W < nwin) {                     // uniform; always true for a full chunk
+            assemble_window<W>(a, e[W], lt);
+            assemble_windows<W + 1>(a, e, nwin, lt);
+        }
     }
-    return pos / 4;
+}
+
+// Number of non-zero elements among a lane's 32: compare + predicated add each.
+__device__ __forceinline__ void count_nonzero(uint32_t& cnt, uint32_t e) {
+    asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p add.u32 %0, %0, 1;\n\t}" : "+r"(cnt) : "r"(e));
 }
 
 // 4-byte elements.  A lane holds one element of each of the chunk's 32 windows
@@ -161,12 +180,15 @@ __device__ __forceinline__ uint32_t assemble_chunk(uint32_t* st, const uint32_t 
 // function whose output the paper offloads, Section IV) and, if relu_out is not
 // null, also writes the dense activation map for the next layer -- the input is
 // read once for both.
-template <typename T, bool RELU>
-__global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
-zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
-                    uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
-                    uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above) {
-    static_assert(sizeof(T) == 4, "2-byte elements have a kernel of their own");
+// FULL: every chunk of the tile has all 1024 elements (true for every tile but
+// possibly the last); the two cases are separate straight-line instantiations so
+// that the common one carries no trace of the ragged one.
+template <bool RELU, bool FULL>
+__device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ src, uint64_t n,
+                                                  uint8_t* __restrict__ dst, uint64_t cap,
+                                                  uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
+                                                  uint32_t num_tiles, uint64_t num_chunks,
+                                                  uint32_t* __restrict__ relu_out, uint32_t tile) {
     constexpr uint32_t S = 4;
     extern __shared__ __align__(16) uint8_t smem_raw[];
     uint32_t* s_tile = reinterpret_cast<uint32_t*>(smem_raw);   // up to kTileChunks * 1056 units
@@ -179,22 +201,13 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     const uint32_t lt = lanemask_lt();
     uint64_t* desc = ws + kWsDescriptors;
 
-    // Tile = block index.  Thread blocks are dispatched in increasing index order,
-    // so every tile this one will wait for belongs to a block that is already
-    // running or finished (the assumption single-pass scans rest on); should it
-    // ever not hold, the bounded wait below turns it into CDMA_ERR_TIMEOUT.
-    const uint32_t tile = blockIdx.x;
-    if (tile >= num_tiles) return;
-    prefetch_future_tile(src, n * S, tile);
-
     // ---- load the warp's chunk: 32 loads per lane, all in flight --------------
     const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunks + warp;
     const uint64_t e0 = chunk * kChunk;
-    uint32_t nwin;   // windows this chunk really has
+    uint32_t nwin = kChunkWindows;   // windows this chunk really has
     uint32_t e[kChunkWindows];
-    if (e0 + kChunk <= n) {
-        nwin = kChunkWindows;
-        const T* p = src + e0 + lane;
+    if (FULL) {
+        const uint32_t* p = src + e0 + lane;
 #pragma unroll
         for (uint32_t w = 0; w < kChunkWindows; ++w) e[w] = __ldcs(p + w * kWindow);
         if (RELU) {
@@ -206,7 +219,7 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
         }
     } else {
         const uint64_t left = (e0 < n) ? (n - e0) : 0;
-        nwin = static_cast<uint32_t>((left + kWindow - 1) / kWindow);
+        nwin = static_cast<uint32_t>(((left < kChunk ? left : kChunk) + kWindow - 1) / kWindow);
 #pragma unroll
         for (uint32_t w = 0; w < kChunkWindows; ++w) {
             const uint64_t j = static_cast<uint64_t>(w) * kWindow + lane;
@@ -221,7 +234,7 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     // ---- 1. count: the tile's size needs only the number of non-zeros ---------
     uint32_t mine = 0;
 #pragma unroll
-    for (uint32_t w = 0; w < kChunkWindows; ++w) mine += (e[w] != 0u) ? 1u : 0u;
+    for (uint32_t w = 0; w < kChunkWindows; ++w) count_nonzero(mine, e[w]);
     const uint32_t units = nwin + __reduce_add_sync(0xffffffffu, mine);
     if (lane == 0) s_chunk_units[warp] = units;
     __syncthreads();
@@ -237,9 +250,9 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     }
 
     // ---- 2. assemble the chunk's records at its place in the staged tile ------
-    uint32_t* st = s_tile + chunk_off;
-    if (nwin == kChunkWindows) assemble_chunk<true>(st, e, nwin, lane, lt);
-    else assemble_chunk<false>(st, e, nwin, lane, lt);
+    // (a recursive template rather than a loop, so that the window number is an immediate)
+    uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(s_tile + chunk_off));
+    assemble_windows<0>(a, e, FULL ? kChunkWindows : nwin, lt);
 
     // ---- 3. the tile's place in the stream ------------------------------------
     if (warp == 0) {
@@ -280,6 +293,25 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     const uint32_t head = min(room, (32u - static_cast<uint32_t>(first_unit & 31u)) & 31u);
     if (threadIdx.x < head) out[threadIdx.x] = s_tile[threadIdx.x];
     for (uint32_t u = head + threadIdx.x; u < room; u += kTileThreads) out[u] = s_tile[u];
+}
+
+template <typename T, bool RELU>
+__global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
+zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
+                    uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
+                    uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above) {
+    static_assert(sizeof(T) == 4, "2-byte elements have a kernel of their own");
+    // Tile = block index.  Thread blocks are dispatched in increasing index order,
+    // so every tile this one will wait for belongs to a block that is already
+    // running or finished (the assumption single-pass scans rest on); should it
+    // ever not hold, the bounded wait in the walk turns it into CDMA_ERR_TIMEOUT.
+    const uint32_t tile = blockIdx.x;
+    if (tile >= num_tiles) return;
+    prefetch_future_tile(src, n * sizeof(T), tile);
+    if ((static_cast<uint64_t>(tile) + 1) * (kTileChunks * kChunk) <= n)
+        compress_tile_u32<RELU, true>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, tile);
+    else
+        compress_tile_u32<RELU, false>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, tile);
 }
 
 // 2-byte elements: the same four steps with 8 consecutive elements per lane (one
