@@ -121,7 +121,34 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
     const uint32_t end = static_cast<uint32_t>(hi - a0) / S;
     bool bad = false;
 
-    if (nelem == kChunk) {
+    if (nelem == kChunk && S == 2) {
+        // full chunk of 2-byte elements: 16 rounds of 2 windows; a half-warp expands a
+        // window, a lane 2 consecutive elements (one 4-byte store per lane, 128
+        // contiguous bytes per warp).  Fewer instructions per element than the 4-byte
+        // scheme below, which matters here: with half the bytes per element this
+        // kernel is bound by instruction issue, not by DRAM.
+        const uint32_t half = lane >> 4;
+        const uint32_t sh = 2u * (lane & 15u);
+        const uint32_t below = (1u << sh) - 1u;
+        uint32_t* out = reinterpret_cast<uint32_t*>(dst + e0) + lane;
+#pragma unroll
+        for (uint32_t g = 0; g < kChunkWindows / 2; ++g) {
+            const uint32_t pa = p;
+            const uint32_t ma = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
+            p += MU + __popc(ma);
+            const uint32_t pb = p;
+            const uint32_t mb = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
+            p += MU + __popc(mb);
+            // a malformed record may carry the walk past the chunk: flag it and pull the
+            // position back (every second round) so that no later read leaves the buffer
+            if (g & 1u) { bad |= (p > end); p = min(p, end); }
+            const uint32_t my_m = half ? mb : ma;
+            const uint32_t q = (half ? pb : pa) + MU + __popc(my_m & below);
+            const uint32_t two = (my_m >> sh) & 3u;
+            const uint32_t v0 = units[q], v1 = units[q + (two & 1u)];
+            __stcs(out + g * 32, ((two & 1u) ? v0 : 0u) | ((two & 2u) ? (v1 << 16) : 0u));
+        }
+    } else if (nelem == kChunk) {
         // full chunk: 8 rounds of 4 windows; lane = 4 consecutive elements
         const uint32_t sub = lane & 7u;
         const uint32_t wj = lane >> 3;
