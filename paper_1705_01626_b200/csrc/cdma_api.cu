@@ -110,7 +110,7 @@ uint64_t cdma_zvc_table_entries(uint64_t n) { return num_chunks_of(n) + 1; }
 
 uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype) {
     (void)dtype;
-    const uint64_t bytes = kWsHeaderBytes + 8 * num_tiles_of(n);
+    const uint64_t bytes = kWsHeaderBytes + 8 * kDescStride * num_tiles_of(n);
     return (bytes + 255) & ~255ull;
 }
 
@@ -134,7 +134,7 @@ static int compress_enqueue(const void* d_src, uint64_t n, int dtype, int layout
     uint64_t* ws = static_cast<uint64_t*>(d_workspace);
 
     // result words and every tile descriptor start at zero
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * num_tiles_of(n), stream) != cudaSuccess)
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * kDescStride * num_tiles_of(n), stream) != cudaSuccess)
         return CDMA_ERR_CUDA;
     if (n == 0) {
         if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return CDMA_ERR_CUDA;

@@ -25,8 +25,8 @@ namespace {
 // Largest tensor the built-in workspace serves: 2^28 elements (1 GiB of fp32).
 constexpr uint64_t kStaticMaxElements = 1ull << 28;
 constexpr uint64_t kStaticWsBytes =
-    (cdma::kWsHeaderBytes + 8 * ((kStaticMaxElements / cdma::kChunk + cdma::kTileChunks - 1) / cdma::kTileChunks) +
-     255) / 256 * 256;                                   // 174,848 bytes
+    (cdma::kWsHeaderBytes + 8 * cdma::kDescStride * ((kStaticMaxElements / cdma::kChunk + cdma::kTileChunks - 1) / cdma::kTileChunks) +
+     255) / 256 * 256;                                   // 699,136 bytes
 
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 
@@ -80,7 +80,7 @@ extern "C" int64_t cdma_zvc_compress_static_ws(const void* d_src, uint64_t n, in
 
     // The array keeps whatever the previous call left: ticket, result words and
     // the descriptors of every tile this call uses must start at zero.
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * num_tiles_of(n), stream) != cudaSuccess)
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * kDescStride * num_tiles_of(n), stream) != cudaSuccess)
         return -static_cast<int64_t>(CDMA_ERR_CUDA);
     if (n == 0) {
         if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return -static_cast<int64_t>(CDMA_ERR_CUDA);

@@ -31,8 +31,15 @@ constexpr uint32_t kWsTicket = 0;      // reserved (tiles are taken in block-ind
 constexpr uint32_t kWsReserved = 1;
 constexpr uint32_t kWsBytes = 2;       // result: payload bytes (compress) / dense bytes (decompress)
 constexpr uint32_t kWsStatus = 3;      // result: first error code, 0 = none
-constexpr uint32_t kWsDescriptors = 4; // one 64-bit prefix descriptor per tile follows
+constexpr uint32_t kWsDescriptors = 4; // prefix descriptors follow, one 64-bit word per tile every kDescStride words
 constexpr uint64_t kWsHeaderBytes = 8 * kWsDescriptors;
+// Descriptors are kDescStride words apart: one per 32-byte sector, so that a tile
+// publishing its descriptor does not contend in L2 with the walks that are
+// reading its neighbours' (packed descriptors cost 10 % of the kernel's time).
+#ifndef CDMA_DESC_STRIDE
+#define CDMA_DESC_STRIDE 4
+#endif
+constexpr uint32_t kDescStride = CDMA_DESC_STRIDE;
 
 // Inter-tile prefix descriptor: {state:2 | value:62} in one 64-bit word so
 // that state and value are published by a single store.

@@ -45,7 +45,7 @@ __device__ LookbackResult lookback_walk(const uint64_t* desc, uint64_t* ws, uint
     while (true) {
         const int64_t idx = look - static_cast<int64_t>(lane);
         // before tile 0 there is nothing: an inclusive prefix of zero
-        const uint64_t d = (idx >= 0) ? ld_relaxed_u64(desc + idx) : kDescPrefix;
+        const uint64_t d = (idx >= 0) ? ld_relaxed_u64(desc + idx * kDescStride) : kDescPrefix;
         const uint32_t state = static_cast<uint32_t>(d >> 62);
         const uint32_t m_prefix = __ballot_sync(0xffffffffu, state == 2);
         const uint32_t m_invalid = __ballot_sync(0xffffffffu, state == 0);
@@ -71,11 +71,16 @@ __device__ LookbackResult lookback_walk(const uint64_t* desc, uint64_t* ws, uint
             if (polls > 2) __nanosleep(100);
             continue;
         }
-        uint64_t v = ((upto >> lane) & 1u) ? (d & kDescValueMask) : 0ull;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        r.exclusive += v;
-        if (m_prefix) break;
+        // A tile is at most 50,688 bytes, so the sizes of up to 32 tiles add up in
+        // 32 bits: one warp reduction; the 64-bit prefix comes from the lane that
+        // holds it.
+        const uint32_t sizes = upto & ~f;                       // lanes holding a size to add
+        const uint32_t part = ((sizes >> lane) & 1u) ? static_cast<uint32_t>(d) : 0u;
+        r.exclusive += __reduce_add_sync(0xffffffffu, part);
+        if (m_prefix) {
+            r.exclusive += __shfl_sync(0xffffffffu, d, __ffs(m_prefix) - 1) & kDescValueMask;
+            break;
+        }
         look -= 32;
     }
     return r;
@@ -246,7 +251,7 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
         tile_bytes = static_cast<uint64_t>(__reduce_add_sync(0xffffffffu, cu)) * S;
         // the tile's size is public before any record is assembled
         if (lane == 0)
-            st_relaxed_u64(desc + tile, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+            st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
     }
 
     // ---- 2. assemble the chunk's records at its place in the staged tile ------
@@ -260,7 +265,7 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
         if (tile != 0) {
             lb = lookback_walk(desc, ws, tile);
             if (lane == 0)
-                st_relaxed_u64(desc + tile, lb.failed ? kDescError
+                st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride, lb.failed ? kDescError
                                                       : (kDescPrefix | (lb.exclusive + tile_bytes)));
         }
         if (lane == 0) {
@@ -422,7 +427,7 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
         if (lane < kTileChunksU16) s_chunk_off[lane] = ci - cu;
         tile_bytes = static_cast<uint64_t>(__shfl_sync(0xffffffffu, ci, kTileChunksU16 - 1)) * S;
         if (lane == 0)
-            st_relaxed_u64(desc + tile, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+            st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
     }
 
     // ---- 2. assemble the records of both chunks in shared memory -------------
@@ -471,7 +476,7 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
         if (tile != 0) {
             lb = lookback_walk(desc, ws, tile);
             if (lane == 0)
-                st_relaxed_u64(desc + tile, lb.failed ? kDescError
+                st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride, lb.failed ? kDescError
                                                       : (kDescPrefix | (lb.exclusive + tile_bytes)));
         }
         if (lane == 0) {
