@@ -169,7 +169,7 @@ int cdma_zvc_relu_compress_async(const void* d_src, uint64_t n, int dtype, int l
  * get offloaded), plug-ins that only ever receive buffers from their host
  * application, start-up and tear-down hooks.  (The paper has no counterpart:
  * its engine needs no software workspace.)  The call takes no workspace; it
- * uses one built into the library, a fixed device array of 699,136 bytes that
+ * uses one built into the library, a fixed device array of 1,048,832 bytes that
  * every GPU loading the library holds until the process exits, and it calls no
  * cudaMalloc, cudaFree or any other allocating routine.
  *

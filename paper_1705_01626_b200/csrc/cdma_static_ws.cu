@@ -26,7 +26,7 @@ namespace {
 constexpr uint64_t kStaticMaxElements = 1ull << 28;
 constexpr uint64_t kStaticWsBytes =
     (cdma::kWsHeaderBytes + 8 * cdma::kDescStride * ((kStaticMaxElements / cdma::kChunk + cdma::kTileChunks - 1) / cdma::kTileChunks) +
-     255) / 256 * 256;                                   // 699,136 bytes
+     255) / 256 * 256;                                   // 1,048,832 bytes
 
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 

@@ -17,10 +17,10 @@ constexpr uint32_t kChunk = kWindow * kChunkWindows;   // 1024 elements
 
 // Compression tiling: one CTA = one tile = kTileChunks chunks, one warp per chunk.
 #ifndef CDMA_TILE_CHUNKS
-#define CDMA_TILE_CHUNKS 12
+#define CDMA_TILE_CHUNKS 8
 #endif
 #ifndef CDMA_MIN_CTAS
-#define CDMA_MIN_CTAS 3
+#define CDMA_MIN_CTAS 5
 #endif
 constexpr uint32_t kTileChunks = CDMA_TILE_CHUNKS;
 constexpr uint32_t kMinCtasPerSm = CDMA_MIN_CTAS;

@@ -2,24 +2,23 @@
 // prefix-sum / shift / append stages of the engine in Section V-B, Fig. 10a).
 //
 // One CTA compresses one tile of kTileChunks chunks; one warp owns one chunk
-// (32 windows of 32 elements).  A lane loads 4 consecutive elements with one
-// vector load, so a warp instruction covers 4 windows (8 lanes per window).
+// (32 windows of 32 elements).  4-byte elements: a lane holds one element of
+// every window, so a window's mask is one warp ballot.  2-byte elements: a lane
+// holds 8 consecutive elements (4 lanes per window, masks by xor-shuffles) and
+// a warp owns two chunks.
 //
 // Order of work inside a CTA, chosen so that the one step that depends on other
 // CTAs (the running byte offset across tiles) waits as little as possible:
-//   1. count: the tile's size needs only the number of non-zeros, so each warp
-//      reduces the pop-count of its "non-zero" nibbles and the tile's size is
-//      published at once, before any record exists;
-//   2. assemble: the 4-bit nibbles of the 8 lanes of a window are OR-combined
-//      with xor-shuffles into the window's 32-bit mask; __popc of the mask bits
-//      below a lane's nibble is the slot of its first value; records go to the
-//      warp's staging area in shared memory;
+//   1. count: the tile's size needs only the number of non-zeros, so it is
+//      reduced and published at once, before any record exists;
+//   2. assemble: mask words and non-zero values go to shared memory; the
+//      pop-count of the mask bits below an element is the slot of its value;
 //   3. look back: warp 0 walks the 64-bit {state,value} descriptors of earlier
 //      tiles (single-pass decoupled look-back, 32 per round); tiles follow the
 //      block index, so a tile only ever waits for blocks dispatched before it;
 //      by now its predecessors have had the whole of step 2 to publish;
-//   4. copy: each warp writes its chunk's bytes to their place in the payload
-//      with coalesced stores.
+//   4. copy: the staged bytes go to their place in the payload with coalesced
+//      stores.
 #include "zvc_common.cuh"
 
 namespace cdma {
@@ -98,14 +97,14 @@ __device__ __forceinline__ void load4(const uint16_t* p, uint32_t (&e)[4]) {
 
 // Tiles follow the block index and blocks are dispatched in that order, so the
 // tile `kPrefetchAhead` places further on will be picked up by a CTA that starts
-// about one CTA lifetime from now (3 CTAs x 148 SMs are resident at a time).
+// about half a CTA lifetime from now (5 CTAs x 148 SMs are resident at a time).
 // Asking L2 for it now turns that CTA's DRAM-latency load phase into L2 hits;
 // every line is still fetched from DRAM exactly once.
 #ifndef CDMA_PREFETCH_AHEAD
-#define CDMA_PREFETCH_AHEAD 444
+#define CDMA_PREFETCH_AHEAD 370
 #endif
 constexpr uint32_t kPrefetchAhead = CDMA_PREFETCH_AHEAD;
-constexpr uint32_t kTileBytes = kTileChunks * kChunk * 4;      // 48 KB for either element width
+constexpr uint32_t kTileBytes = kTileChunks * kChunk * 4;      // 32 KB for either element width
 
 __device__ __forceinline__ void prefetch_future_tile(const void* src, uint64_t total_bytes, uint32_t tile) {
     if (kPrefetchAhead == 0) return;
@@ -321,7 +320,7 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
 
 // 2-byte elements: the same four steps with 8 consecutive elements per lane (one
 // 16-byte load), so a warp instruction covers 8 windows (4 lanes per window), and
-// two chunks per warp, so that a tile is as many bytes (48 KB) as in the 4-byte
+// two chunks per warp, so that a tile is as many bytes (32 KB) as in the 4-byte
 // kernel and the look-back runs at the same rate per byte.
 constexpr uint32_t kTileChunksU16 = 2 * kTileChunks;
 
