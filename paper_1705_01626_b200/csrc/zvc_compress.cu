@@ -199,6 +199,7 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
     __shared__ uint32_t s_chunk_units[kTileChunks];
     __shared__ uint64_t s_base;
     __shared__ uint32_t s_failed;
+    __shared__ uint32_t s_room;
 
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
@@ -270,12 +271,15 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
         if (lane == 0) {
             s_base = lb.exclusive;
             s_failed = lb.failed ? 1u : 0u;
+            // units of this tile that fit below the capacity
+            const uint64_t end_bytes = lb.exclusive + tile_bytes;
+            s_room = static_cast<uint32_t>((cap >= end_bytes ? tile_bytes : (cap > lb.exclusive ? cap - lb.exclusive : 0)) / S);
             if (!lb.failed) {
                 if (tile == num_tiles - 1) {
-                    table[num_chunks] = lb.exclusive + tile_bytes;
-                    ws[kWsBytes] = lb.exclusive + tile_bytes;
+                    table[num_chunks] = end_bytes;
+                    ws[kWsBytes] = end_bytes;
                 }
-                if (lb.exclusive + tile_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
+                if (end_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
             }
         }
     }
@@ -285,13 +289,7 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
     // ---- 4. the CTA writes the tile's bytes to their place, below cap ---------
     const uint64_t first_unit = s_base / S;
     if (lane == 0 && chunk < num_chunks) table[chunk] = (first_unit + chunk_off) * S;
-    uint32_t tile_units = 0;                                    // same sum in every warp
-#pragma unroll
-    for (uint32_t c = 0; c < kTileChunks; ++c) tile_units += s_chunk_units[c];
-    const uint64_t cap_units = cap / S;
-    const uint32_t room = (first_unit >= cap_units) ? 0u
-                        : (cap_units - first_unit < tile_units ? static_cast<uint32_t>(cap_units - first_unit)
-                                                               : tile_units);
+    const uint32_t room = s_room;
     uint32_t* out = reinterpret_cast<uint32_t*>(dst) + first_unit;
     // units in front of the first 128-byte line boundary of the destination
     const uint32_t head = min(room, (32u - static_cast<uint32_t>(first_unit & 31u)) & 31u);
