@@ -290,11 +290,25 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
     const uint64_t first_unit = s_base / S;
     if (lane == 0 && chunk < num_chunks) table[chunk] = (first_unit + chunk_off) * S;
     const uint32_t room = s_room;
-    uint32_t* out = reinterpret_cast<uint32_t*>(dst) + first_unit;
-    // units in front of the first 128-byte line boundary of the destination
-    const uint32_t head = min(room, (32u - static_cast<uint32_t>(first_unit & 31u)) & 31u);
-    if (threadIdx.x < head) out[threadIdx.x] = s_tile[threadIdx.x];
-    for (uint32_t u = head + threadIdx.x; u < room; u += kTileThreads) out[u] = s_tile[u];
+    // Row r of the copy is the aligned 128-byte line r of the destination that the
+    // tile touches: thread t moves unit u = t - mis + r * kTileThreads, where mis is
+    // how far the tile's first unit sits inside its line; only row 0 can have u < 0.
+    const uint32_t mis = static_cast<uint32_t>(first_unit) & 31u;
+    const uint32_t* sp = s_tile + threadIdx.x - mis;            // never dereferenced below s_tile
+    uint32_t* gp = reinterpret_cast<uint32_t*>(dst) + first_unit + threadIdx.x - mis;
+    int32_t left = static_cast<int32_t>(room) + static_cast<int32_t>(mis) - static_cast<int32_t>(threadIdx.x);
+    // `left` > 0 <=> this thread's unit of the current row is below the end of the tile
+    if (threadIdx.x >= mis && left > 0) *gp = *sp;
+    left -= kTileThreads; sp += kTileThreads; gp += kTileThreads;
+    while (left > 3 * static_cast<int32_t>(kTileThreads)) {
+        const uint32_t v0 = sp[0], v1 = sp[kTileThreads], v2 = sp[2 * kTileThreads], v3 = sp[3 * kTileThreads];
+        gp[0] = v0; gp[kTileThreads] = v1; gp[2 * kTileThreads] = v2; gp[3 * kTileThreads] = v3;
+        left -= 4 * kTileThreads; sp += 4 * kTileThreads; gp += 4 * kTileThreads;
+    }
+    while (left > 0) {
+        *gp = *sp;
+        left -= kTileThreads; sp += kTileThreads; gp += kTileThreads;
+    }
 }
 
 template <typename T, bool RELU>
