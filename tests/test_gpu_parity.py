@@ -12,7 +12,7 @@ import torch
 from oracle import zvc_c, zvc_numpy
 from paper_1705_01626_b200 import binding as B
 from paper_1705_01626_b200 import workloads as wl
-from tests.gpu_helpers import DeviceCodec, raw_numpy
+from tests.gpu_helpers import CANARY, DeviceCodec, raw_numpy
 
 pytestmark = pytest.mark.gpu
 
@@ -124,6 +124,30 @@ def test_capacity_too_small_is_reported_without_overrun():
         assert codec.payload_numpy(cap).tobytes() == want[:cap].tobytes()
     codec = DeviceCodec(x.numel(), x.dtype, capacity=(len(want) + 15) & ~15)
     assert codec.compress(x) == len(want)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+def test_capacity_at_tile_and_line_boundaries(dtype):
+    """Capacities that end on, just before and just after the places where the copy-out
+    changes row or tile: everything below the capacity is the stream's prefix, nothing
+    above it is touched."""
+    x, raw = make(5 * TILE + 3 * 1024 + 41, 0.45, 17, dtype)
+    want, table = zvc_c.compress(raw)
+    s = x.element_size()
+    tile_starts = [int(table[k]) for k in range(0, len(table) - 1, 8)]      # first chunk of every 8th
+    caps = set()
+    for t in tile_starts[1:4]:
+        line = (t + 127) // 128 * 128                                       # first full line of the tile
+        for c in (t - s, t, t + s, line - s, line, line + s, line + 128 * 8 + 4 * s, t + 10):
+            if 0 <= c < len(want):
+                caps.add(c)
+    for cap in sorted(caps):
+        codec = DeviceCodec(x.numel(), x.dtype, capacity=cap)
+        assert codec.compress(x) == -B.ERR_BUFFER_TOO_SMALL
+        assert codec.canaries_intact()
+        whole = cap // s * s                                                # whole elements below the capacity
+        assert codec.payload_numpy(whole).tobytes() == want[:whole].tobytes(), cap
+        assert (codec.payload_numpy(cap)[whole:] == CANARY).all(), cap
 
 
 def test_corrupt_table_and_stream_are_rejected_without_faulting():
