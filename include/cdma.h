@@ -299,11 +299,17 @@ int cdma_ticket_host_view(cdma_ctx* ctx, cdma_ticket ticket, const void** h_payl
                           const uint64_t** h_table);
 
 /*
- * The same compressed copies for callers whose tensors live in HOST memory
- * (pinned for full speed): h_src is copied to the device, compressed, and the
- * payload and table copied back into h_dst / h_table; and the reverse.  They
- * run on the context's side stream, wait for completion and return C / n*s.
- * h_table holds cdma_zvc_table_entries(n) uint64.
+ * The same compressed copies for callers whose tensors live in HOST memory.
+ * When all three buffers are page-locked (cudaHostAlloc / cudaHostRegister,
+ * tensor and payload 16-byte aligned) a single kernel reads the source over
+ * the host link and writes the result back over it as it goes -- the software
+ * form of the paper's one compressed-copy call (Section V-D), both directions
+ * of the link busy at once and no device staging.  Otherwise h_src is copied
+ * to the device, processed there and the result copied back.  Both run on the
+ * context's side stream, wait for completion and return C / n*s.
+ * h_table holds cdma_zvc_table_entries(n) uint64.  On CDMA_ERR_BUFFER_TOO_SMALL
+ * the page-locked path may already have written payload bytes below
+ * dst_capacity (never beyond it); the staged path leaves h_dst untouched.
  */
 int64_t cdma_zvc_compress_host(cdma_ctx* ctx, const void* h_src, uint64_t n, int dtype,
                                int layout, void* h_dst, uint64_t dst_capacity,

@@ -44,6 +44,16 @@ static cudaError_t enqueue_result(const uint64_t* ws, uint64_t* h_result, cudaSt
     return cudaMemcpyAsync(h_result, ws + kWsBytes, 16, cudaMemcpyDeviceToHost, stream);
 }
 
+// True when p lies in page-locked host memory (which kernels reach over the host link).
+static bool in_host_memory(const void* p) {
+    cudaPointerAttributes attr;
+    if (p == nullptr || cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    return attr.type == cudaMemoryTypeHost;
+}
+
 static inline bool aligned(const void* p, uintptr_t a) {
     return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0;
 }
@@ -139,10 +149,12 @@ static int compress_enqueue(const void* d_src, uint64_t n, int dtype, int layout
     if (n == 0) {
         if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return CDMA_ERR_CUDA;
     } else {
+        const bool on_device = !in_host_memory(d_src);
         const uint32_t nan_above = (dtype == CDMA_F32) ? 0x7f800000u : (dtype == CDMA_F16 ? 0x7c00u : 0x7f80u);
         const cudaError_t e =
-            relu ? launch_zvc_relu_compress(d_src, n, s, nan_above, d_relu_out, d_dst, dst_capacity, d_table, ws, stream)
-                 : launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, stream);
+            relu ? launch_zvc_relu_compress(d_src, n, s, nan_above, d_relu_out, d_dst, dst_capacity, d_table, ws, stream,
+                                            on_device)
+                 : launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, stream, on_device);
         if (e != cudaSuccess) return CDMA_ERR_CUDA;
     }
     if (enqueue_result(ws, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
@@ -207,7 +219,7 @@ int cdma_zvc_decompress_async(const void* d_src, uint64_t src_bytes, const uint6
     uint64_t* ws = static_cast<uint64_t*>(d_workspace);
 
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return CDMA_ERR_CUDA;
-    if (launch_zvc_decompress(d_src, src_bytes, d_table, n, s, d_dst, ws, stream) != cudaSuccess)
+    if (launch_zvc_decompress(d_src, src_bytes, d_table, n, s, d_dst, ws, stream, !in_host_memory(d_src)) != cudaSuccess)
         return CDMA_ERR_CUDA;
     if (enqueue_result(ws, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
     return CDMA_OK;

@@ -129,6 +129,19 @@ bool plan_slot(const Slot& slot, uint64_t n, int dtype, SlotPlan* p) {
     return true;
 }
 
+// Device view of a page-locked host buffer (mapped into the device's address space
+// under unified addressing), or nullptr if p is anything else or not aligned to `align`.
+void* mapped_view(const void* p, uintptr_t align) {
+    cudaPointerAttributes attr;
+    if (p == nullptr || cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) return nullptr;
+    if (reinterpret_cast<uintptr_t>(attr.devicePointer) & (align - 1)) return nullptr;
+    return attr.devicePointer;
+}
+
 uint64_t* next_result_words(cdma_ctx* ctx) {
     uint64_t* r = ctx->h_results + 2 * (ctx->next_result % kResultRing);
     ++ctx->next_result;
@@ -466,7 +479,32 @@ int64_t cdma_zvc_compress_host(cdma_ctx* ctx, const void* h_src, uint64_t n, int
         return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
     const uint32_t s = cdma_dtype_size(dtype);
     if (s == 0) return -static_cast<int64_t>(CDMA_ERR_UNSUPPORTED_DTYPE);
-    int st = ensure_dense(ctx, n * s);
+    int st;
+    {
+        // All three buffers page-locked: one kernel reads the tensor and writes payload and
+        // table over the host link as it goes (both directions of the link busy at once),
+        // with no device staging and no separate copies.
+        void* m_src = n ? mapped_view(h_src, 16) : nullptr;
+        void* m_dst = dst_capacity ? mapped_view(h_dst, 16) : nullptr;
+        void* m_table = mapped_view(h_table, 8);
+        if ((n == 0 || m_src) && (dst_capacity == 0 || m_dst) && m_table) {
+            Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
+            SlotPlan p;
+            if (!plan_slot(slot, n, dtype, &p)) return -static_cast<int64_t>(CDMA_ERR_BUFFER_TOO_SMALL);
+            if (slot.used && cudaStreamWaitEvent(ctx->side, slot.idle, 0) != cudaSuccess)
+                return -static_cast<int64_t>(CDMA_ERR_CUDA);
+            uint64_t* res = next_result_words(ctx);
+            st = cdma_zvc_compress_async(m_src, n, dtype, layout, m_dst, dst_capacity,
+                                         static_cast<uint64_t*>(m_table), p.ws, p.ws_bytes, ctx->side, res);
+            if (st != CDMA_OK) return -static_cast<int64_t>(st);
+            slot.used = true;
+            cudaEventRecord(slot.idle, ctx->side);
+            if (cudaStreamSynchronize(ctx->side) != cudaSuccess) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+            if (res[1] != 0) return -static_cast<int64_t>(res[1]);
+            return static_cast<int64_t>(res[0]);
+        }
+    }
+    st = ensure_dense(ctx, n * s);
     if (st != CDMA_OK) return -static_cast<int64_t>(st);
     Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
     SlotPlan p;
@@ -503,7 +541,31 @@ int64_t cdma_zvc_decompress_host(cdma_ctx* ctx, const void* h_src, uint64_t src_
         return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
     const uint32_t s = cdma_dtype_size(dtype);
     if (s == 0) return -static_cast<int64_t>(CDMA_ERR_UNSUPPORTED_DTYPE);
-    int st = ensure_dense(ctx, n * s);
+    int st;
+    {
+        // All three buffers page-locked: one kernel loads payload and table over the host
+        // link and stores the dense tensor back over it.
+        void* m_src = src_bytes ? mapped_view(h_src, 16) : nullptr;
+        void* m_table = mapped_view(h_table, 8);
+        void* m_dst = n ? mapped_view(h_dst, 16) : nullptr;
+        if ((src_bytes == 0 || m_src) && (n == 0 || m_dst) && m_table) {
+            Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
+            SlotPlan p;
+            if (!plan_slot(slot, n, dtype, &p)) return -static_cast<int64_t>(CDMA_ERR_BUFFER_TOO_SMALL);
+            if (slot.used && cudaStreamWaitEvent(ctx->side, slot.idle, 0) != cudaSuccess)
+                return -static_cast<int64_t>(CDMA_ERR_CUDA);
+            uint64_t* res = next_result_words(ctx);
+            st = cdma_zvc_decompress_async(m_src, src_bytes, static_cast<const uint64_t*>(m_table), n, dtype,
+                                           layout, m_dst, p.ws, p.ws_bytes, ctx->side, res);
+            if (st != CDMA_OK) return -static_cast<int64_t>(st);
+            slot.used = true;
+            cudaEventRecord(slot.idle, ctx->side);
+            if (cudaStreamSynchronize(ctx->side) != cudaSuccess) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+            if (res[1] != 0) return -static_cast<int64_t>(res[1]);
+            return static_cast<int64_t>(n * s);
+        }
+    }
+    st = ensure_dense(ctx, n * s);
     if (st != CDMA_OK) return -static_cast<int64_t>(st);
     Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
     SlotPlan p;

@@ -83,16 +83,18 @@ __device__ __forceinline__ void report_status(uint64_t* ws, uint32_t code) {
               static_cast<unsigned long long>(code));
 }
 
-// Launchers (defined next to their kernels).  elem_size is 2 or 4.
+// Launchers (defined next to their kernels).  elem_size is 2 or 4.  src_on_device
+// is false when the input lies in mapped host memory: the kernels then leave out
+// their L2 prefetches, which would fetch every line over the host link twice.
 cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst,
                                 uint64_t cap, uint64_t* d_table, uint64_t* d_ws,
-                                cudaStream_t stream);
+                                cudaStream_t stream, bool src_on_device = true);
 cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
                                      void* d_relu_out, void* d_dst, uint64_t cap, uint64_t* d_table,
-                                     uint64_t* d_ws, cudaStream_t stream);
+                                     uint64_t* d_ws, cudaStream_t stream, bool src_on_device = true);
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, bool src_on_device = true);
 void count_kernel_launch();
 void timing_before_launch(cudaStream_t stream);   // measurement hook, see cdma_time_next_kernel
 void timing_after_launch(cudaStream_t stream);

@@ -315,7 +315,8 @@ template <typename T, bool RELU>
 __global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
 zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
                     uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
-                    uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above) {
+                    uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above,
+                    uint64_t prefetch_bytes) {
     static_assert(sizeof(T) == 4, "2-byte elements have a kernel of their own");
     // Tile = block index.  Thread blocks are dispatched in increasing index order,
     // so every tile this one will wait for belongs to a block that is already
@@ -323,7 +324,7 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     // ever not hold, the bounded wait in the walk turns it into CDMA_ERR_TIMEOUT.
     const uint32_t tile = blockIdx.x;
     if (tile >= num_tiles) return;
-    prefetch_future_tile(src, n * sizeof(T), tile);
+    prefetch_future_tile(src, prefetch_bytes, tile);
     if ((static_cast<uint64_t>(tile) + 1) * (kTileChunks * kChunk) <= n)
         compress_tile_u32<RELU, true>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, tile);
     else
@@ -341,7 +342,7 @@ __global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
 zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst,
                         uint64_t cap, uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
                         uint32_t num_tiles, uint64_t num_chunks, uint16_t* __restrict__ relu_out,
-                        uint32_t nan_above) {
+                        uint32_t nan_above, uint64_t prefetch_bytes) {
     using T = uint16_t;
     constexpr uint32_t S = 2, MU = 2;
     constexpr uint32_t kMaxChunkUnits = MU * kChunkWindows + kChunk;
@@ -360,7 +361,7 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
     uint64_t* desc = ws + kWsDescriptors;
     const uint32_t tile = blockIdx.x;     // block-index order, as in the 4-byte kernel
     if (tile >= num_tiles) return;
-    prefetch_future_tile(src, n * S, tile);
+    prefetch_future_tile(src, prefetch_bytes, tile);
 
     // ---- load the warp's two chunks ------------------------------------------
     uint32_t nwin[2];
@@ -523,7 +524,7 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
 template <typename T, uint32_t TILE_CHUNKS, typename Kernel>
 cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_dst, uint64_t cap,
                          uint64_t* d_table, uint64_t* d_ws, void* d_relu_out, uint32_t nan_above,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, bool src_on_device) {
     constexpr uint32_t kSmem = TILE_CHUNKS * (4 * kChunkWindows + sizeof(T) * kChunk);
     const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
@@ -532,7 +533,8 @@ cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_d
     timing_before_launch(stream);
     kernel<<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
         static_cast<const T*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
-        static_cast<uint32_t>(tiles), chunks, static_cast<T*>(d_relu_out), nan_above);
+        static_cast<uint32_t>(tiles), chunks, static_cast<T*>(d_relu_out), nan_above,
+        src_on_device ? n * sizeof(T) : 0ull);
     timing_after_launch(stream);
     return cudaGetLastError();
 }
@@ -541,28 +543,28 @@ cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_d
 
 cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst,
                                 uint64_t cap, uint64_t* d_table, uint64_t* d_ws,
-                                cudaStream_t stream) {
+                                cudaStream_t stream, bool src_on_device) {
     if (num_tiles_of(n) == 0) return cudaSuccess;
     const cudaError_t e =
         (elem_size == 4)
             ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t, false>, d_src, n, d_dst, cap,
-                                                  d_table, d_ws, nullptr, 0, stream)
+                                                  d_table, d_ws, nullptr, 0, stream, src_on_device)
             : launch_typed<uint16_t, kTileChunksU16>(zvc_compress_kernel_u16<false>, d_src, n, d_dst, cap,
-                                                     d_table, d_ws, nullptr, 0, stream);
+                                                     d_table, d_ws, nullptr, 0, stream, src_on_device);
     count_kernel_launch();
     return e;
 }
 
 cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
                                      void* d_relu_out, void* d_dst, uint64_t cap, uint64_t* d_table,
-                                     uint64_t* d_ws, cudaStream_t stream) {
+                                     uint64_t* d_ws, cudaStream_t stream, bool src_on_device) {
     if (num_tiles_of(n) == 0) return cudaSuccess;
     const cudaError_t e =
         (elem_size == 4)
             ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t, true>, d_src, n, d_dst, cap,
-                                                  d_table, d_ws, d_relu_out, nan_above, stream)
+                                                  d_table, d_ws, d_relu_out, nan_above, stream, src_on_device)
             : launch_typed<uint16_t, kTileChunksU16>(zvc_compress_kernel_u16<true>, d_src, n, d_dst, cap,
-                                                     d_table, d_ws, d_relu_out, nan_above, stream);
+                                                     d_table, d_ws, d_relu_out, nan_above, stream, src_on_device);
     count_kernel_launch();
     return e;
 }

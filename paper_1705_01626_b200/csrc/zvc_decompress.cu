@@ -205,14 +205,14 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
 
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, bool src_on_device) {
     const uint64_t chunks = num_chunks_of(n);
     if (chunks == 0) return cudaSuccess;
     const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
     timing_before_launch(stream);
     if (elem_size == 4) {
         // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
-        const bool prefetch = src_bytes >= (n * 4) / 5;
+        const bool prefetch = src_on_device && src_bytes >= (n * 4) / 5;
         auto kernel = prefetch ? zvc_decompress_kernel<uint32_t, true> : zvc_decompress_kernel<uint32_t, false>;
         kernel<<<grid, kDecThreads, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes, d_table, n,
                                                  static_cast<uint32_t*>(d_dst), d_ws, chunks);

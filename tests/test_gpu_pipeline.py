@@ -108,16 +108,20 @@ def test_pool_exhaustion_and_small_staging_are_reported():
         B.cdma_ctx_destroy(ctx)
 
 
+@pytest.mark.parametrize("pinned", [True, False])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
-def test_host_buffer_calls_match_the_oracle(dtype):
+def test_host_buffer_calls_match_the_oracle(dtype, pinned):
+    """Page-locked buffers take the one-kernel path (the kernel reads and writes host
+    memory directly); pageable ones are staged through device memory."""
     n = 300_000 + 77
     code = B.F32 if dtype == torch.float32 else B.F16
-    x = wl.iid_relu_like((n,), 0.3, seed=8, device="cpu", dtype=dtype, floor=2.0 ** -10).pin_memory()
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    x = pin(wl.iid_relu_like((n,), 0.3, seed=8, device="cpu", dtype=dtype, floor=2.0 ** -10))
     cap = B.cdma_zvc_max_compressed_bytes(n, code)
     entries = B.cdma_zvc_table_entries(n)
-    h_p = torch.zeros(cap, dtype=torch.uint8).pin_memory()
-    h_t = torch.zeros(entries, dtype=torch.int64).pin_memory()
-    h_y = torch.zeros(n, dtype=dtype).pin_memory()
+    h_p = pin(torch.zeros(cap, dtype=torch.uint8))
+    h_t = pin(torch.zeros(entries, dtype=torch.int64))
+    h_y = pin(torch.zeros(n, dtype=dtype))
     ctx = B.cdma_ctx_create(1 << 16, 2 * (cap + 8 * entries + B.cdma_zvc_workspace_bytes(n, code) + 4096))
     try:
         c = B.cdma_zvc_compress_host(ctx, x.data_ptr(), n, code, B.NCHW, h_p.data_ptr(), cap, h_t.data_ptr())
@@ -132,7 +136,7 @@ def test_host_buffer_calls_match_the_oracle(dtype):
         assert B.cdma_zvc_compress_host(ctx, x.data_ptr(), n, code, B.NCHW, h_p.data_ptr(), c - 4,
                                         h_t.data_ptr()) == -B.ERR_BUFFER_TOO_SMALL
         # a corrupted table is reported, not followed
-        bad = h_t.clone().pin_memory()
+        bad = pin(h_t.clone())
         bad[1] += 4
         assert B.cdma_zvc_decompress_host(ctx, h_p.data_ptr(), c, bad.data_ptr(), n, code, B.NCHW,
                                           h_y.data_ptr()) == -B.ERR_CORRUPT_STREAM
