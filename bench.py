@@ -793,6 +793,105 @@ def run_relu(args):
                             "fused_payload_only": (dense + c) / t_f / 1e6 / peak}}), flush=True)
 
 
+def run_timeline(args):
+    """Training-step estimate of Section VI's model, fed with numbers measured on this GPU: forward and
+    backward time of the 13 conv layers of a VGG-16-shaped CNN (batch 64, torch's convolution, used for
+    timing only), the codec's time and ratio on each layer's synthetic activation map (the config3 set),
+    and the pinned-copy rates of the host link."""
+    import torch
+    import torch.nn.functional as F
+    from paper_1705_01626_b200 import binding as B
+    from paper_1705_01626_b200 import timeline as tl
+    from paper_1705_01626_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    batch = 64
+    g = torch.Generator(device="cuda").manual_seed(BASE_SEED_RELU + 1)
+
+    def timed(fn, iters=5):
+        for _ in range(2):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters * 1e-3
+
+    # host link, pinned, 1 GiB each way
+    hbuf = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
+    dbuf = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+    d2h = (1 << 30) / timed(lambda: hbuf.copy_(dbuf, non_blocking=True)) / 1e9
+    h2d = (1 << 30) / timed(lambda: dbuf.copy_(hbuf, non_blocking=True)) / 1e9
+    del hbuf, dbuf
+    link = min(d2h, h2d)
+
+    rows, plain, packed = [], [], []
+    cin = 3
+    prev = None                        # (bytes, ratio, compress_s, decompress_s) of the map feeding this layer
+    for i, (cout, h, w) in enumerate(wl.VGG16_CONV_SHAPES):
+        x = torch.randn(batch, cin, h, w, generator=g, device=dev).requires_grad_(True)
+        wt = (torch.randn(cout, cin, 3, 3, generator=g, device=dev) * 0.05).requires_grad_(True)
+        gy = torch.randn(batch, cout, h, w, generator=g, device=dev)
+        fwd = timed(lambda: F.relu(F.conv2d(x, wt, padding=1)))
+        y = F.relu(F.conv2d(x, wt, padding=1))
+        bwd = timed(lambda: torch.autograd.grad(y, (x, wt), gy, retain_graph=True))
+        del y, gy, wt
+        # the map saved for this layer's backward pass: the input images for the first layer, else the
+        # previous conv + ReLU output (before any pooling, as in the config3 set)
+        if prev is None:
+            act_bytes, ratio, t_c, t_d = batch * cin * h * w * 4, 1.0, 0.0, 0.0
+        else:
+            act_bytes, ratio, t_c, t_d = prev[:4]
+        del x
+        rows.append({"layer": i, "fwd_ms": fwd * 1e3, "bwd_ms": bwd * 1e3, "input_map_MB": act_bytes / 1e6,
+                     "ratio": ratio, "plain_copy_ms": act_bytes / (link * 1e9) * 1e3,
+                     "compressed_copy_ms": act_bytes / ratio / (link * 1e9) * 1e3,
+                     "compress_ms": t_c * 1e3, "decompress_ms": t_d * 1e3})
+        plain.append(tl.Layer(fwd, bwd, act_bytes, 1.0))
+        packed.append((fwd, bwd, act_bytes, ratio, t_c, t_d))
+        # this layer's output map: synthetic stand-in with the config3 recipe, through the codec
+        d = 0.5 - 0.4 * i / (len(wl.VGG16_CONV_SHAPES) - 1)
+        a = wl.correlated_relu((batch, cout, h, w), d, wl.seed_for(3, i), dev)
+        c, ms_c, ms_d = time_codec(B, a, B.F32, iters=5)
+        nbytes = a.numel() * 4
+        prev = (nbytes, nbytes / (c + 8 * B.cdma_zvc_table_entries(a.numel())), ms_c * 1e-3, ms_d * 1e-3)
+        del a
+        cin = cout
+        torch.cuda.empty_cache()
+    # software codec: compression runs on the GPU in front of the copy (added to the layer that produces the
+    # copy's overlap window), decompression of the map a layer below needs runs beside the layer above it
+    cdma = []
+    for i, (fwd, bwd, act_bytes, ratio, t_c, t_d) in enumerate(packed):
+        t_d_above = packed[i - 1][5] if i > 0 else 0.0
+        cdma.append(tl.Layer(fwd + t_c, bwd + t_d_above, act_bytes, ratio))
+
+    def both(pcie, dram):
+        sp = tl.summary(plain, pcie)
+        sc = tl.summary(cdma, pcie, dram)
+        return {"pcie_GBps": pcie, "oracle_ms": sp["oracle_s"] * 1e3, "vdnn_ms": sp["vdnn_s"] * 1e3,
+                "cdma_ms": sc["cdma_s"] * 1e3, "vdnn_vs_oracle": sp["vdnn_vs_oracle"],
+                "cdma_vs_oracle": sp["oracle_s"] / sc["cdma_s"],
+                "cdma_speedup_over_vdnn": sp["vdnn_s"] / sc["cdma_s"],
+                "traffic_reduction": sc["traffic_reduction"], "max_comp_bw_GBps": sc["max_comp_bw_gbs"]}
+
+    peak, _ = measured_peak()
+    print(json.dumps({
+        "workload": "timeline: 13 conv layers of a VGG-16-shaped CNN, batch 64, fp32 tensors (TF32 convolutions), "
+                    "config3 activation maps",
+        "model": "Section VI: copy time = bytes / ratio / PCIe x max(1, ratio x PCIe / DRAM_BW); "
+                 "a layer stalls when its copy outlasts it",
+        "link": {"d2h_GBps": d2h, "h2d_GBps": h2d},
+        "layers": rows,
+        "this_box": both(link, peak),
+        "same_layers_on_a_16_GBps_link": both(16.0, peak),
+        "paper_context": "paper (Titan X, PCIe gen3, six CNNs): vDNN loses 31 % on average, compressed copies win "
+                         "back 32 % on average (61 % at most)",
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -814,6 +913,8 @@ def main():
         run_sweep(args)
     elif args.workload == "relu":
         run_relu(args)
+    elif args.workload == "timeline":
+        run_timeline(args)
     else:
         run_cdma(args)
 
