@@ -150,20 +150,21 @@ def test_capacity_at_tile_and_line_boundaries(dtype):
         assert (codec.payload_numpy(cap)[whole:] == CANARY).all(), cap
 
 
-def test_corrupt_table_and_stream_are_rejected_without_faulting():
-    x, raw = make(4 * TILE + 300, 0.4, 11, torch.float32)
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+def test_corrupt_table_and_stream_are_rejected_without_faulting(dtype):
+    x, raw = make(4 * TILE + 300, 0.4, 11, dtype)
     n = x.numel()
     payload, table = zvc_c.compress(raw)
-    out = torch.zeros(n, dtype=torch.float32, device="cuda")
+    out = torch.zeros(n, dtype=dtype, device="cuda")
 
     def run(p, t, nbytes=None):
-        codec = DeviceCodec(n, torch.float32)
+        codec = DeviceCodec(n, dtype)
         codec.load(p, t)
         r = codec.decompress(out, len(p) if nbytes is None else nbytes)
         assert codec.canaries_intact()
         return r
 
-    assert run(payload, table) == 4 * n
+    assert run(payload, table) == x.element_size() * n
     t = table.copy(); t[3] += 4
     assert run(payload, t) == -B.ERR_CORRUPT_STREAM
     t = table.copy(); t[5] = t[4] - 4                       # decreasing offsets
@@ -178,9 +179,12 @@ def test_corrupt_table_and_stream_are_rejected_without_faulting():
     last_mask = int(zvc_numpy.window_offsets(raw)[2 * 32 - 1])
     p[last_mask] ^= 0x10
     assert run(p, table) == -B.ERR_CORRUPT_STREAM
-    with pytest.raises(ValueError):
-        zvc_c.decompress(p, n, np.float32)
+    if dtype == torch.float32:     # (the table-less serial walk of the oracle can fall back into step on 2-byte data)
+        with pytest.raises(ValueError):
+            zvc_c.decompress(p, n, np.float32)
     assert run(payload, table, nbytes=len(payload) - 4) == -B.ERR_CORRUPT_STREAM
+    if dtype != torch.float32:
+        return
     # a mask naming an element beyond n (short last window)
     y, rawy = make(40, 1.0, 1, torch.float32)
     py, ty = zvc_c.compress(rawy)
@@ -188,6 +192,47 @@ def test_corrupt_table_and_stream_are_rejected_without_faulting():
     codec = DeviceCodec(40, torch.float32)
     codec.load(bad, ty)
     assert codec.decompress(torch.zeros(40, device="cuda"), len(bad)) == -B.ERR_CORRUPT_STREAM
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+def test_garbage_streams_never_fault(dtype):
+    """Streams that are not streams: random bytes, all-ones masks (records as long as they get),
+    zeros, behind tables whose chunk sizes are possible.  The answer is CORRUPT_STREAM (or, by
+    luck, success); nothing is read outside the payload or written outside the tensor."""
+    n = 6 * 1024 + 500
+    s = torch.empty(0, dtype=dtype).element_size()
+    k = (n + 1023) // 1024
+    rng = np.random.default_rng(170501626)
+    guard = 64
+    for trial in range(16):
+        sizes = []
+        for c in range(k):
+            nelem = min(1024, n - 1024 * c)
+            nwin = (nelem + 31) // 32
+            lo, hi = 4 * nwin, 4 * nwin + s * nelem
+            pick = [lo, hi, (lo + hi) // 2, int(rng.integers(lo, hi + 1))][trial % 4]
+            sizes.append(pick // s * s)
+        table = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+        total = int(table[-1])
+        kind = (trial // 4) % 4
+        if kind == 0:
+            payload = rng.integers(0, 256, size=total, dtype=np.uint8)
+        elif kind == 1:
+            payload = np.full(total, 0xFF, dtype=np.uint8)
+        elif kind == 2:
+            payload = np.zeros(total, dtype=np.uint8)
+        else:
+            payload = rng.integers(0, 2, size=total, dtype=np.uint8) * 0xFF
+        codec = DeviceCodec(n, dtype)
+        codec.load(payload, table)
+        out = torch.full((n + guard,), 7.0, dtype=dtype, device="cuda")
+        r = codec.decompress(out, total)
+        assert r in (-B.ERR_CORRUPT_STREAM, n * s), B.status_string(r)
+        assert codec.canaries_intact()
+        assert bool((out[n:] == 7.0).all())
+    # the library still works afterwards
+    x, raw = make(n, 0.3, 2, dtype)
+    check_against_oracle(x, raw)
 
 
 def test_argument_checks():
