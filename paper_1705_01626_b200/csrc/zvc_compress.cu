@@ -331,49 +331,108 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
         compress_tile_u32<RELU, false>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, tile);
 }
 
-// 2-byte elements: the same four steps with 8 consecutive elements per lane (one
-// 16-byte load), so a warp instruction covers 8 windows (4 lanes per window), and
-// two chunks per warp, so that a tile is as many bytes (32 KB) as in the 4-byte
-// kernel and the look-back runs at the same rate per byte.
+// 2-byte elements: a lane holds 8 consecutive elements (one 16-byte load), so a
+// warp instruction covers 8 windows (4 lanes per window), and a warp owns two
+// chunks, so that a tile is as many bytes (32 KB) as in the 4-byte kernel.  The
+// steps are the same; masks come from xor-shuffles over the 4 lanes of a window,
+// record positions from a shuffle-up scan over the 8 windows of a group.  The
+// inner pieces are blocks of PTX for the same reason as in the 4-byte kernel:
+// with half the bytes per element this kernel is bound by instruction issue.
 constexpr uint32_t kTileChunksU16 = 2 * kTileChunks;
+constexpr uint32_t kGroupsU16 = kChunk / 256;                   // 256 elements per warp load
 
-template <bool RELU>
-__global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
-zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst,
-                        uint64_t cap, uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
-                        uint32_t num_tiles, uint64_t num_chunks, uint16_t* __restrict__ relu_out,
-                        uint32_t nan_above, uint64_t prefetch_bytes) {
-    using T = uint16_t;
-    constexpr uint32_t S = 2, MU = 2;
-    constexpr uint32_t kMaxChunkUnits = MU * kChunkWindows + kChunk;
-    constexpr uint32_t kGroups = kChunk / 256;                  // 256 elements per warp load
-    extern __shared__ __align__(16) uint8_t smem_raw[];
-    T (*stage)[kMaxChunkUnits] = reinterpret_cast<T (*)[kMaxChunkUnits]>(smem_raw);
+// "Non-zero" flags of the two halves of w, or-ed into bits at LO and HI.
+template <uint32_t LO, uint32_t HI>
+__device__ __forceinline__ void flag_pair_u16(uint32_t& bits, uint32_t w) {
+    asm("{\n\t.reg .pred p, q;\n\t.reg .b32 t;\n\t"
+        "and.b32 t, %1, 0xffff;\n\tsetp.ne.u32 p, t, 0;\n\t@p or.b32 %0, %0, %2;\n\t"
+        "setp.gt.u32 q, %1, 0xffff;\n\t@q or.b32 %0, %0, %3;\n\t}"
+        : "+r"(bits) : "r"(w), "n"(LO), "n"(HI));
+}
+
+// Append the non-zero halves of w (low half first) at shared byte address q + 4
+// (q points at the window's mask word), advancing q by 2 per value stored.
+__device__ __forceinline__ void append_pair_u16(uint32_t& q, uint32_t w) {
+    asm volatile("{\n\t.reg .pred p, r;\n\t.reg .b32 t;\n\t.reg .b16 l, h;\n\t"
+                 "mov.b32 {l, h}, %1;\n\t"
+                 "and.b32 t, %1, 0xffff;\n\tsetp.ne.u32 p, t, 0;\n\t"
+                 "@p st.shared.u16 [%0+4], l;\n\t@p add.u32 %0, %0, 2;\n\t"
+                 "setp.gt.u32 r, %1, 0xffff;\n\t"
+                 "@r st.shared.u16 [%0+4], h;\n\t@r add.u32 %0, %0, 2;\n\t}"
+                 : "+r"(q) : "r"(w) : "memory");
+}
+
+// A 32-bit mask word at a 2-byte aligned shared address, by the lanes with `on` set
+// (predicated stores, no branch in front of the next shuffles).
+__device__ __forceinline__ void sts_mask_u16(uint32_t saddr, uint32_t v, uint32_t on) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b16 l, h;\n\tsetp.ne.u32 p, %2, 0;\n\tmov.b32 {l, h}, %1;\n\t"
+                 "@p st.shared.u16 [%0], l;\n\t@p st.shared.u16 [%0+2], h;\n\t}"
+                 ::"r"(saddr), "r"(v), "r"(on) : "memory");
+}
+
+// Records of one chunk from its 32 flag bits per lane and the lane's 32 elements;
+// `a` = shared byte address where the chunk's records start.  FULL: all 32
+// windows exist; otherwise only the first nwin do (elements past the end were
+// loaded as zeros, so only their mask records have to be suppressed).
+template <bool FULL>
+__device__ __forceinline__ void assemble_chunk_u16(uint32_t a, uint32_t bits, const uint32_t (&w)[kGroupsU16][4],
+                                                   uint32_t lane, uint32_t nwin) {
+    const uint32_t sub = lane & 3u;                       // which byte of the window's mask is mine
+    const uint32_t below = (1u << (8u * sub)) - 1u;
+    const uint32_t first = sub == 0u ? 1u : 0u;
+#pragma unroll
+    for (uint32_t g = 0; g < kGroupsU16; ++g) {
+        uint32_t m = ((bits >> (8u * g)) & 0xffu) << (8u * sub);
+        m |= __shfl_xor_sync(0xffffffffu, m, 1);
+        m |= __shfl_xor_sync(0xffffffffu, m, 2);           // the window's 32-bit mask
+        const bool live = FULL || (8u * g + (lane >> 2)) < nwin;
+        const uint32_t rec = live ? 4u + 2u * __popc(m) : 0u;   // record length in bytes, same in 4 lanes
+        uint32_t incl = rec;
+        uint32_t t = __shfl_up_sync(0xffffffffu, incl, 4);
+        if (lane >= 4) incl += t;
+        t = __shfl_up_sync(0xffffffffu, incl, 8);
+        if (lane >= 8) incl += t;
+        t = __shfl_up_sync(0xffffffffu, incl, 16);
+        if (lane >= 16) incl += t;                          // records of windows up to mine
+        const uint32_t mine = a + incl - rec;               // where my window's record starts
+        a += __shfl_sync(0xffffffffu, incl, 31);
+        sts_mask_u16(mine, m, (FULL || live) ? first : 0u);
+        uint32_t q = mine + 2u * __popc(m & below);
+        append_pair_u16(q, w[g][0]);
+        append_pair_u16(q, w[g][1]);
+        append_pair_u16(q, w[g][2]);
+        append_pair_u16(q, w[g][3]);
+    }
+}
+
+template <bool RELU, bool FULL>
+__device__ __forceinline__ void compress_tile_u16(const uint16_t* __restrict__ src, uint64_t n,
+                                                  uint8_t* __restrict__ dst, uint64_t cap,
+                                                  uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
+                                                  uint32_t num_tiles, uint64_t num_chunks,
+                                                  uint16_t* __restrict__ relu_out, uint32_t nan_above,
+                                                  uint32_t tile) {
+    constexpr uint32_t S = 2;
+    extern __shared__ __align__(16) uint8_t smem_raw[];          // the tile's records, contiguous
     __shared__ uint32_t s_chunk_units[kTileChunksU16];
-    __shared__ uint32_t s_chunk_off[kTileChunksU16];
     __shared__ uint64_t s_base;
     __shared__ uint32_t s_failed;
+    __shared__ uint32_t s_room;
 
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
-    const uint32_t sub = lane & 3u;       // position of this lane's byte in its window's mask
-    const uint32_t wj = lane >> 2;        // which of the 8 windows of a group
     uint64_t* desc = ws + kWsDescriptors;
-    const uint32_t tile = blockIdx.x;     // block-index order, as in the 4-byte kernel
-    if (tile >= num_tiles) return;
-    prefetch_future_tile(src, prefetch_bytes, tile);
 
     // ---- load the warp's two chunks ------------------------------------------
-    uint32_t nwin[2];
-    uint32_t w[2][kGroups][4];            // 8 elements of a group = 4 words of two halves
+    uint32_t nwin[2] = {kChunkWindows, kChunkWindows};
+    uint32_t w[2][kGroupsU16][4];         // 8 elements of a group = 4 words of two halves
 #pragma unroll
     for (uint32_t c = 0; c < 2; ++c) {
         const uint64_t e0 = (static_cast<uint64_t>(tile) * kTileChunksU16 + 2 * warp + c) * kChunk;
-        if (e0 + kChunk <= n) {
-            nwin[c] = kChunkWindows;
-            const T* p = src + e0 + 8 * lane;
+        if (FULL) {
+            const uint16_t* p = src + e0 + 8 * lane;
 #pragma unroll
-            for (uint32_t g = 0; g < kGroups; ++g) {
+            for (uint32_t g = 0; g < kGroupsU16; ++g) {
                 const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p + g * 256));
                 w[c][g][0] = q.x; w[c][g][1] = q.y; w[c][g][2] = q.z; w[c][g][3] = q.w;
                 if (RELU) {
@@ -388,9 +447,9 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
             }
         } else {
             const uint64_t left = (e0 < n) ? (n - e0) : 0;
-            nwin[c] = static_cast<uint32_t>((left + kWindow - 1) / kWindow);
+            nwin[c] = static_cast<uint32_t>(((left < kChunk ? left : kChunk) + kWindow - 1) / kWindow);
 #pragma unroll
-            for (uint32_t g = 0; g < kGroups; ++g) {
+            for (uint32_t g = 0; g < kGroupsU16; ++g) {
 #pragma unroll
                 for (uint32_t k = 0; k < 4; ++k) {
                     const uint64_t j = static_cast<uint64_t>(g) * 256 + 8 * lane + 2 * k;
@@ -399,8 +458,8 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
                     if (RELU) {
                         lo = relu_bits16(lo, nan_above);
                         hi = relu_bits16(hi, nan_above);
-                        if (relu_out != nullptr && j < left) relu_out[e0 + j] = static_cast<T>(lo);
-                        if (relu_out != nullptr && j + 1 < left) relu_out[e0 + j + 1] = static_cast<T>(hi);
+                        if (relu_out != nullptr && j < left) relu_out[e0 + j] = static_cast<uint16_t>(lo);
+                        if (relu_out != nullptr && j + 1 < left) relu_out[e0 + j + 1] = static_cast<uint16_t>(hi);
                     }
                     w[c][g][k] = lo | (hi << 16);
                 }
@@ -408,79 +467,39 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
         }
     }
 
-    // ---- 1. count: 8 "non-zero" bits per group, 4 groups packed in one word --
-    uint32_t bits[2];
+    // ---- 1. count: 8 "non-zero" bits per group, 4 groups in one word -----------
+    uint32_t bits[2] = {0u, 0u};
+    uint32_t units[2];
 #pragma unroll
     for (uint32_t c = 0; c < 2; ++c) {
-        bits[c] = 0;
-#pragma unroll
-        for (uint32_t g = 0; g < kGroups; ++g) {
-            uint32_t b8 = 0;
-#pragma unroll
-            for (uint32_t k = 0; k < 4; ++k) {
-                b8 |= ((w[c][g][k] & 0xffffu) != 0u ? 1u : 0u) << (2 * k);
-                b8 |= ((w[c][g][k] >> 16) != 0u ? 2u : 0u) << (2 * k);
-            }
-            bits[c] |= b8 << (8 * g);
-        }
-        const uint32_t units = MU * nwin[c] + __reduce_add_sync(0xffffffffu, __popc(bits[c]));
-        if (lane == 0) s_chunk_units[2 * warp + c] = units;
+        flag_pair_u16<1u << 0, 1u << 1>(bits[c], w[c][0][0]);   flag_pair_u16<1u << 2, 1u << 3>(bits[c], w[c][0][1]);
+        flag_pair_u16<1u << 4, 1u << 5>(bits[c], w[c][0][2]);   flag_pair_u16<1u << 6, 1u << 7>(bits[c], w[c][0][3]);
+        flag_pair_u16<1u << 8, 1u << 9>(bits[c], w[c][1][0]);   flag_pair_u16<1u << 10, 1u << 11>(bits[c], w[c][1][1]);
+        flag_pair_u16<1u << 12, 1u << 13>(bits[c], w[c][1][2]); flag_pair_u16<1u << 14, 1u << 15>(bits[c], w[c][1][3]);
+        flag_pair_u16<1u << 16, 1u << 17>(bits[c], w[c][2][0]); flag_pair_u16<1u << 18, 1u << 19>(bits[c], w[c][2][1]);
+        flag_pair_u16<1u << 20, 1u << 21>(bits[c], w[c][2][2]); flag_pair_u16<1u << 22, 1u << 23>(bits[c], w[c][2][3]);
+        flag_pair_u16<1u << 24, 1u << 25>(bits[c], w[c][3][0]); flag_pair_u16<1u << 26, 1u << 27>(bits[c], w[c][3][1]);
+        flag_pair_u16<1u << 28, 1u << 29>(bits[c], w[c][3][2]); flag_pair_u16<1u << 30, 1u << 31>(bits[c], w[c][3][3]);
+        units[c] = 2 * nwin[c] + __reduce_add_sync(0xffffffffu, __popc(bits[c]));
+        if (lane == 0) s_chunk_units[2 * warp + c] = units[c];
     }
     __syncthreads();
+    // every warp sums the chunks in front of its own; warp 0 also needs the total
+    const uint32_t cu = (lane < kTileChunksU16) ? s_chunk_units[lane] : 0u;
+    const uint32_t chunk_off = __reduce_add_sync(0xffffffffu, lane < 2 * warp ? cu : 0u);
     uint64_t tile_bytes = 0;
     if (warp == 0) {
-        const uint32_t cu = (lane < kTileChunksU16) ? s_chunk_units[lane] : 0u;
-        uint32_t ci = cu;
-#pragma unroll
-        for (int o = 1; o < static_cast<int>(kTileChunksU16); o <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xffffffffu, ci, o);
-            if (lane >= static_cast<uint32_t>(o)) ci += t;
-        }
-        if (lane < kTileChunksU16) s_chunk_off[lane] = ci - cu;
-        tile_bytes = static_cast<uint64_t>(__shfl_sync(0xffffffffu, ci, kTileChunksU16 - 1)) * S;
+        tile_bytes = static_cast<uint64_t>(__reduce_add_sync(0xffffffffu, cu)) * S;
+        // the tile's size is public before any record is assembled
         if (lane == 0)
-            st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+            st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride,
+                           (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
     }
 
-    // ---- 2. assemble the records of both chunks in shared memory -------------
-    uint32_t run[2];
-    const uint32_t below = (1u << (8 * sub)) - 1u;
-#pragma unroll
-    for (uint32_t c = 0; c < 2; ++c) {
-        T* st = stage[2 * warp + c];
-        uint32_t r = 0;
-#pragma unroll
-        for (uint32_t g = 0; g < kGroups; ++g) {
-            const uint32_t b8 = (bits[c] >> (8 * g)) & 0xffu;
-            uint32_t m = b8 << (8 * sub);
-            m |= __shfl_xor_sync(0xffffffffu, m, 1);
-            m |= __shfl_xor_sync(0xffffffffu, m, 2);           // the window's 32-bit mask
-            const bool live = (g * 8 + wj) < nwin[c];
-            const uint32_t rec = live ? (MU + __popc(m)) : 0u;
-            uint32_t incl = rec;
-            uint32_t t = __shfl_up_sync(0xffffffffu, incl, 4);
-            if (lane >= 4) incl += t;
-            t = __shfl_up_sync(0xffffffffu, incl, 8);
-            if (lane >= 8) incl += t;
-            t = __shfl_up_sync(0xffffffffu, incl, 16);
-            if (lane >= 16) incl += t;                         // records of windows <= wj
-            const uint32_t pos = r + incl - rec;
-            r += __shfl_sync(0xffffffffu, incl, 31);
-            if (live) {
-                if (sub == 0) {
-                    st[pos] = static_cast<T>(m & 0xffffu);
-                    st[pos + 1] = static_cast<T>(m >> 16);
-                }
-                uint32_t q = pos + MU + __popc(m & below);
-#pragma unroll
-                for (uint32_t k = 0; k < 4; ++k) {
-                    if (b8 & (1u << (2 * k))) st[q++] = static_cast<T>(w[c][g][k] & 0xffffu);
-                    if (b8 & (2u << (2 * k))) st[q++] = static_cast<T>(w[c][g][k] >> 16);
-                }
-            }
-        }
-        run[c] = r;
-    }
+    // ---- 2. assemble both chunks' records at their place in the staged tile ----
+    const uint32_t s_addr = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw));
+    assemble_chunk_u16<FULL>(s_addr + S * chunk_off, bits[0], w[0], lane, nwin[0]);
+    assemble_chunk_u16<FULL>(s_addr + S * (chunk_off + units[0]), bits[1], w[1], lane, nwin[1]);
 
     // ---- 3. the tile's place in the stream ------------------------------------
     if (warp == 0) {
@@ -488,37 +507,79 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
         if (tile != 0) {
             lb = lookback_walk(desc, ws, tile);
             if (lane == 0)
-                st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride, lb.failed ? kDescError
-                                                      : (kDescPrefix | (lb.exclusive + tile_bytes)));
+                st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride,
+                               lb.failed ? kDescError : (kDescPrefix | (lb.exclusive + tile_bytes)));
         }
         if (lane == 0) {
             s_base = lb.exclusive;
             s_failed = lb.failed ? 1u : 0u;
+            // bytes of this tile that fit below the capacity (whole units)
+            const uint64_t end_bytes = lb.exclusive + tile_bytes;
+            s_room = static_cast<uint32_t>((cap >= end_bytes ? tile_bytes : (cap > lb.exclusive ? cap - lb.exclusive : 0)) / S) * S;
             if (!lb.failed) {
                 if (tile == num_tiles - 1) {
-                    table[num_chunks] = lb.exclusive + tile_bytes;
-                    ws[kWsBytes] = lb.exclusive + tile_bytes;
+                    table[num_chunks] = end_bytes;
+                    ws[kWsBytes] = end_bytes;
                 }
-                if (lb.exclusive + tile_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
+                if (end_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
             }
         }
     }
     __syncthreads();
     if (s_failed) return;
 
-    // ---- 4. each warp writes its chunks' bytes to their place, below cap ------
-    const uint64_t cap_units = cap / S;
-#pragma unroll
-    for (uint32_t c = 0; c < 2; ++c) {
-        const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunksU16 + 2 * warp + c;
-        const uint64_t first_unit = s_base / S + s_chunk_off[2 * warp + c];
-        if (lane == 0 && chunk < num_chunks) table[chunk] = first_unit * S;
-        T* out = reinterpret_cast<T*>(dst) + first_unit;
-        const T* st = stage[2 * warp + c];
-        const uint32_t room = (first_unit >= cap_units) ? 0u
-                            : (cap_units - first_unit < run[c] ? static_cast<uint32_t>(cap_units - first_unit) : run[c]);
-        for (uint32_t i = lane; i < room; i += 32) out[i] = st[i];
+    // ---- 4. the CTA writes the tile's bytes to their place, below cap ---------
+    const uint64_t base = s_base;
+    if (lane < 2) {
+        const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunksU16 + 2 * warp + lane;
+        if (chunk < num_chunks) table[chunk] = base + S * (chunk_off + (lane ? units[0] : 0u));
     }
+    const uint32_t room = s_room;                                   // bytes, whole units
+    // The payload is only 2-byte aligned.  A halfword in front brings the destination
+    // to a 4-byte boundary; the body goes out as 32-bit words, each warp store one
+    // aligned 128-byte line; a halfword may remain at the end.  When the head halfword
+    // exists the staged words straddle two shared-memory words: funnel shift.
+    const uint32_t hb = (static_cast<uint32_t>(base) & 2u) ? min(2u, room) : 0u;
+    const uint32_t nw = (room - hb) / 4u;
+    const uint32_t tb = room - hb - 4u * nw;                        // 0 or 2 bytes behind the body
+    const uint16_t* s16 = reinterpret_cast<const uint16_t*>(smem_raw);
+    if (threadIdx.x == 0 && hb) *reinterpret_cast<uint16_t*>(dst + base) = s16[0];
+    if (threadIdx.x == 32 && tb) *reinterpret_cast<uint16_t*>(dst + base + hb + 4ull * nw) = s16[(hb + 4u * nw) / 2u];
+    const uint64_t body = base + hb;                                // 4-byte aligned
+    const uint32_t mis = static_cast<uint32_t>(body >> 2) & 31u;    // first word's place in its 128-byte line
+    const uint32_t* sp = reinterpret_cast<const uint32_t*>(smem_raw) + threadIdx.x - mis;
+    uint32_t* gp = reinterpret_cast<uint32_t*>(dst + body) + threadIdx.x - mis;
+    int32_t left = static_cast<int32_t>(nw) + static_cast<int32_t>(mis) - static_cast<int32_t>(threadIdx.x);
+    if (hb == 0) {
+        if (threadIdx.x >= mis && left > 0) *gp = *sp;
+        left -= kTileThreads; sp += kTileThreads; gp += kTileThreads;
+        while (left > 0) {
+            *gp = *sp;
+            left -= kTileThreads; sp += kTileThreads; gp += kTileThreads;
+        }
+    } else {
+        if (threadIdx.x >= mis && left > 0) *gp = __funnelshift_r(sp[0], sp[1], 16);
+        left -= kTileThreads; sp += kTileThreads; gp += kTileThreads;
+        while (left > 0) {
+            *gp = __funnelshift_r(sp[0], sp[1], 16);
+            left -= kTileThreads; sp += kTileThreads; gp += kTileThreads;
+        }
+    }
+}
+
+template <bool RELU>
+__global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
+zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst,
+                        uint64_t cap, uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
+                        uint32_t num_tiles, uint64_t num_chunks, uint16_t* __restrict__ relu_out,
+                        uint32_t nan_above, uint64_t prefetch_bytes) {
+    const uint32_t tile = blockIdx.x;     // block-index order, as in the 4-byte kernel
+    if (tile >= num_tiles) return;
+    prefetch_future_tile(src, prefetch_bytes, tile);
+    if ((static_cast<uint64_t>(tile) + 1) * (kTileChunksU16 * kChunk) <= n)
+        compress_tile_u16<RELU, true>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, nan_above, tile);
+    else
+        compress_tile_u16<RELU, false>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, nan_above, tile);
 }
 
 template <typename T, uint32_t TILE_CHUNKS, typename Kernel>
