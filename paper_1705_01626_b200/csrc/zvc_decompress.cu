@@ -33,22 +33,91 @@ __device__ __forceinline__ void store4(uint16_t* p, uint32_t a, uint32_t b, uint
     __stcs(reinterpret_cast<uint2*>(p), make_uint2(a | (b << 16), c | (d << 16)));
 }
 
+// Shared-memory loads by 32-bit address + immediate: positions in the staged
+// array are kept as byte addresses so that no index has to be scaled.
+template <uint32_t IMM>
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(IMM));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t v;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(v) : "r"(a), "r"(b), "r"(sel));   // the low 16 bits of sel are used
+    return v;
+}
+
+// Per-lane constants of the 4-byte expansion.
+struct U32Lane {
+    uint32_t sh;         // 4 * (lane & 7): where my 4 mask bits start
+    uint32_t below;      // mask bits of the elements in front of mine
+    uint32_t off;        // 4 * (lane >> 3) + 4: my window's place in the round, past its mask word
+    bool w_hi, w_odd;    // bits of lane >> 3
+};
+
+// One round = windows 4G .. 4G+3 of a full chunk of 4-byte elements.  `a` is the
+// shared byte address of the next mask word minus 4 bytes per window already
+// passed (folded into the immediates).  The walk is pulled back to the chunk's
+// end after every second window, so that nothing is read beyond the staged bytes
+// plus two records; a walk that was pulled back once overshoots again at every
+// later step, so the caller only has to look at the last one.
+template <uint32_t G>
+__device__ __forceinline__ void expand_round_u32(uint32_t& a, uint32_t a_end, uint32_t& last, const U32Lane& c,
+                                                 uint4* __restrict__ out) {
+    // four serial steps of the self-delimiting walk; every lane sees all four
+    const uint32_t a0 = a;
+    const uint32_t m0 = lds32<16 * G + 0>(a0);
+    const uint32_t a1 = a0 + 4u * __popc(m0);
+    const uint32_t m1 = lds32<16 * G + 4>(a1);
+    const uint32_t a2 = min(a1 + 4u * __popc(m1), a_end - (16u * G + 8u));
+    const uint32_t m2 = lds32<16 * G + 8>(a2);
+    const uint32_t a3 = a2 + 4u * __popc(m2);
+    const uint32_t m3 = lds32<16 * G + 12>(a3);
+    last = a3 + 4u * __popc(m3);
+    a = min(last, a_end - (16u * G + 16u));
+    const uint32_t my_a = c.w_hi ? (c.w_odd ? a3 : a2) : (c.w_odd ? a1 : a0);
+    const uint32_t my_m = c.w_hi ? (c.w_odd ? m3 : m2) : (c.w_odd ? m1 : m0);
+    // the next four values in front of my elements
+    const uint32_t q = my_a + 4u * __popc(my_m & c.below) + c.off;
+    const uint32_t v0 = lds32<16 * G + 0>(q), v1 = lds32<16 * G + 4>(q), v2 = lds32<16 * G + 8>(q),
+                   v3 = lds32<16 * G + 12>(q);
+    // element k takes the value numbered by the set bits below bit k
+    const uint32_t nib = my_m >> c.sh;
+    const bool b0 = nib & 1u, b1 = nib & 2u, b2 = nib & 4u, b3 = nib & 8u;
+    const uint32_t t1 = b0 ? v1 : v0, u = b0 ? v2 : v1, w = b0 ? v3 : v2;
+    const uint32_t t2 = b1 ? u : t1, x = b1 ? w : u;
+    const uint32_t t3 = b2 ? x : t2;
+    __stcs(out + 32 * G, make_uint4(b0 ? v0 : 0u, b1 ? t1 : 0u, b2 ? t2 : 0u, b3 ? t3 : 0u));
+}
+
+template <uint32_t G>
+__device__ __forceinline__ void expand_rounds_u32(uint32_t& a, uint32_t a_end, uint32_t& last, const U32Lane& c,
+                                                  uint4* __restrict__ out) {
+    if constexpr (G < kChunkWindows / 4) {
+        expand_round_u32<G>(a, a_end, last, c, out);
+        expand_rounds_u32<G + 1>(a, a_end, last, c, out);
+    }
+}
+
 template <typename T, bool PREFETCH>
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, 6)
 zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
                       const uint64_t* __restrict__ table, uint64_t n, T* __restrict__ dst,
                       uint64_t* __restrict__ ws, uint64_t num_chunks) {
     constexpr uint32_t S = sizeof(T);
     constexpr uint32_t MU = 4 / S;                               // units of T per mask
     constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
+    static_assert(S == 4, "2-byte elements have a kernel of their own");
     // 16-byte phase in front; behind, room for the reads of a walk that has left
-    // a malformed record.  4-byte elements: the position is pulled back to `end`
-    // after every window (one more instruction per window, but the smaller buffer
-    // lets a sixth CTA fit per SM); 2-byte elements: after every group of 4
-    // windows, so the walk can run 4 records past `end`.  Either way a lane then
-    // reads a mask and up to 35 values from there.
-    constexpr bool kClampEveryWindow = (S == 4);
-    constexpr uint32_t kOverrun = kClampEveryWindow ? 0u : 4u * (MU + 32u);
+    // a malformed record: the position is pulled back to `end` after every second
+    // window (the buffer then still lets six CTAs fit per SM), so the walk can run
+    // 2 records past `end`, and a lane reads a mask and up to 35 values from there.
+    constexpr uint32_t kOverrun = 2u * (MU + 32u);
     constexpr uint32_t kBuf = (kMaxChunkBytes + 16 + S * (kOverrun + MU + 36) + 15) / 16 * 16;
     static_assert(kBuf % 16 == 0, "rows of s_buf must keep 16-byte alignment for the vector stores");
     __shared__ __align__(16) uint8_t s_buf[kDecWarps][kBuf];
@@ -123,35 +192,17 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
 
     if (nelem == kChunk) {
         // full chunk: 8 rounds of 4 windows; lane = 4 consecutive elements
-        const uint32_t sub = lane & 7u;
-        const uint32_t wj = lane >> 3;
-        const uint32_t below = (1u << (4 * sub)) - 1u;
-        T* out = dst + e0 + 4 * lane;
-#pragma unroll
-        for (uint32_t g = 0; g < kChunk / 128; ++g) {
-            // four serial steps of the self-delimiting walk; every lane sees all four
-            uint32_t pw[4], mw[4];
-#pragma unroll
-            for (uint32_t j = 0; j < 4; ++j) {
-                pw[j] = p;
-                if (S == 4) mw[j] = units[p];
-                else mw[j] = static_cast<uint32_t>(units[p]) | (static_cast<uint32_t>(units[p + 1]) << 16);
-                p += MU + __popc(mw[j]);
-                // a malformed record may carry the walk past the chunk: flag it and pull
-                // the position back so that no later read leaves the staged bytes
-                if (kClampEveryWindow) { bad |= (p > end); p = min(p, end); }
-            }
-            if (!kClampEveryWindow) { bad |= (p > end); p = min(p, end); }
-            const uint32_t my_p = (wj == 0) ? pw[0] : (wj == 1) ? pw[1] : (wj == 2) ? pw[2] : pw[3];
-            const uint32_t my_m = (wj == 0) ? mw[0] : (wj == 1) ? mw[1] : (wj == 2) ? mw[2] : mw[3];
-            const uint32_t nib = (my_m >> (4 * sub)) & 15u;
-            const uint32_t q = my_p + MU + __popc(my_m & below);
-            // element k takes the value numbered by the set bits below bit k
-            const uint32_t c1 = nib & 1u, c2 = __popc(nib & 3u), c3 = __popc(nib & 7u);
-            const uint32_t a0v = units[q], a1v = units[q + c1], a2v = units[q + c2], a3v = units[q + c3];
-            store4(out + g * 128, (nib & 1u) ? a0v : 0u, (nib & 2u) ? a1v : 0u, (nib & 4u) ? a2v : 0u,
-                   (nib & 8u) ? a3v : 0u);
-        }
+        U32Lane c;
+        c.sh = 4u * (lane & 7u);
+        c.below = (1u << c.sh) - 1u;
+        c.off = 4u * (lane >> 3) + 4u;
+        c.w_hi = (lane & 16u) != 0u;
+        c.w_odd = (lane & 8u) != 0u;
+        const uint32_t t_addr = static_cast<uint32_t>(__cvta_generic_to_shared(buf));
+        uint32_t a = t_addr + 4u * p, last = 0;
+        expand_rounds_u32<0>(a, t_addr + 4u * end, last, c, reinterpret_cast<uint4*>(dst + e0) + lane);
+        // `last` is the final position before it was pulled back, with 4 bytes per window folded out
+        p = (last - t_addr) / 4u + kChunkWindows;
     } else {
         // ragged last chunk: lane = element, one window per round
         const uint32_t lt = lanemask_lt();
@@ -186,25 +237,6 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
 // lane's 4 mask bits, so two byte-permute instructions with selectors from a
 // 16-entry table (plus one AND that clears the places of zero elements) do the
 // whole expansion; one 8-byte store per lane, 256 contiguous bytes per warp.
-// Shared-memory loads by 32-bit address + immediate: positions in the staged
-// array are kept as byte addresses so that no index has to be scaled.
-template <uint32_t IMM>
-__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(IMM));
-    return v;
-}
-__device__ __forceinline__ uint2 lds64(uint32_t addr) {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t v;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(v) : "r"(a), "r"(b), "r"(sel));   // the low 16 bits of sel are used
-    return v;
-}
-
 // Per-lane constants of the 2-byte expansion.
 struct U16Lane {
     uint32_t sh;         // 4 * (lane & 7): where my 4 mask bits start
