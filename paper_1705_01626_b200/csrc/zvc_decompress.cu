@@ -176,9 +176,14 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
         if (cf < num_chunks) {
             const uint64_t flo = __ldg(table + cf);
             const uint64_t fhi = __ldg(table + cf + 1);
-            if (flo <= fhi && fhi <= src_bytes && fhi - flo <= kMaxChunkBytes) {
-                for (uint64_t a = (flo & ~127ull) + 128ull * lane; a < fhi; a += 128ull * 32)
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src + a));
+            // at most 34 lines of 128 bytes: one per lane, a second one for the first lanes
+            const uint64_t line0 = flo & ~127ull;
+            const uint64_t span = fhi - line0;                 // garbage if the entries are bad: checked next
+            if (flo <= fhi && fhi <= src_bytes && span <= kMaxChunkBytes + 127) {
+                const uint32_t off = 128u * lane;
+                if (off < static_cast<uint32_t>(span)) asm volatile("prefetch.global.L2 [%0];" ::"l"(src + line0 + off));
+                if (off + 4096u < static_cast<uint32_t>(span))
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src + line0 + off + 4096u));
             }
         }
     }
@@ -380,9 +385,12 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
         if (cf < num_chunks) {
             const uint64_t flo = __ldg(table + cf);
             const uint64_t fhi = __ldg(table + cf + 1);
-            if (flo <= fhi && fhi <= src_bytes && fhi - flo <= 2 * kU16MaxUnits) {
-                for (uint64_t a = (flo & ~127ull) + 128ull * lane; a < fhi; a += 128ull * 32)
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src + a));
+            // at most 18 lines of 128 bytes: one per lane
+            const uint64_t line0 = flo & ~127ull;
+            const uint64_t span = fhi - line0;                 // garbage if the entries are bad: checked next
+            if (flo <= fhi && fhi <= src_bytes && span <= 2 * kU16MaxUnits + 127) {
+                if (128u * lane < static_cast<uint32_t>(span))
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src + line0 + 128u * lane));
             }
         }
     }
