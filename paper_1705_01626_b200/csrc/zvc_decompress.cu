@@ -293,6 +293,17 @@ __device__ __forceinline__ void expand_rounds_u16(uint32_t& a, uint32_t a_end, b
 constexpr uint32_t kU16MaxUnits = 2 * kChunkWindows + kChunk;          // 1088
 constexpr uint32_t kU16Overrun = 4 * (2 + 32);                         // the walk is pulled back every 4 windows
 constexpr uint32_t kU16Entries = (kU16MaxUnits + 8 + kU16Overrun + 2 + 36 + 7) / 8 * 8;
+// Expansion table of the 2-byte kernel, indexed by a lane's 4 mask bits:
+// {sel0 | sel1 << 16, keep1}.  Element k takes value number popc(bits below k);
+// with v01 / v23 the next four values, elements 0,1 = prmt(v01, 0, sel0) (selector
+// nibble 4 picks a zero byte) and elements 2,3 = prmt(v01, v23, sel1) & keep1.
+__constant__ uint2 kExpandU16[16] = {
+    {0x10104444u, 0x00000000u}, {0x32324410u, 0x00000000u}, {0x32321044u, 0x00000000u}, {0x54543210u, 0x00000000u},
+    {0x32104444u, 0x0000ffffu}, {0x54324410u, 0x0000ffffu}, {0x54321044u, 0x0000ffffu}, {0x76543210u, 0x0000ffffu},
+    {0x10104444u, 0xffff0000u}, {0x32324410u, 0xffff0000u}, {0x32321044u, 0xffff0000u}, {0x54543210u, 0xffff0000u},
+    {0x32104444u, 0xffffffffu}, {0x54324410u, 0xffffffffu}, {0x54321044u, 0xffffffffu}, {0x76543210u, 0xffffffffu},
+};
+
 // t[] takes 5 KB per warp, so shared memory allows 44 warps per SM: 11 CTAs of 4 warps.
 #ifndef CDMA_DEC16_WARPS
 #define CDMA_DEC16_WARPS 4
@@ -312,22 +323,8 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
                           uint64_t* __restrict__ ws, uint64_t num_chunks) {
     constexpr uint32_t S = 2, MU = 2;
     __shared__ __align__(32) uint32_t s_t[kDec16Warps][kU16Entries];
-    // Per 4-bit mask: {sel0 | sel1 << 16, keep1}.  Element k takes value number
-    // popc(bits below k).  out0 = prmt(v01, 0, sel0) (nibble 4 picks a zero byte),
-    // out1 = prmt(v01, v23, sel1) & keep1.
     __shared__ uint2 s_expand[16];
-    if (threadIdx.x < 16) {
-        const uint32_t nib = threadIdx.x;
-        uint32_t sel = 0, keep = 0;
-        for (uint32_t k = 0; k < 4; ++k) {
-            const uint32_t r = __popc(nib & ((1u << k) - 1u));              // which value
-            const bool set = (nib >> k) & 1u;
-            const uint32_t lo = (k < 2 && !set) ? 4u : 2u * r, hi = (k < 2 && !set) ? 4u : 2u * r + 1u;
-            sel |= (lo | (hi << 4)) << (8 * k);                             // k = 0,1 -> sel0; k = 2,3 -> sel1
-            if (k >= 2 && set) keep |= 0xffffu << (16 * (k - 2));
-        }
-        s_expand[nib] = make_uint2(sel, keep);
-    }
+    if (threadIdx.x < 16) s_expand[threadIdx.x] = kExpandU16[threadIdx.x];
     __syncthreads();
 
     const uint32_t lane = lane_id();
@@ -343,8 +340,11 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
     // ---- the chunk's byte range, validated ----------------------------------
     const uint64_t lo = __ldg(table + chunk);
     const uint64_t hi = __ldg(table + chunk + 1);
-    bool ok = (lo <= hi) && (hi <= src_bytes) && (hi - lo >= 4ull * nwin) &&
-              (hi - lo <= 4ull * nwin + static_cast<uint64_t>(S) * nelem) && (((lo | hi) & 1ull) == 0);
+    const uint64_t len64 = hi - lo;
+    const uint32_t len = static_cast<uint32_t>(len64);                      // trusted only once len64 is known small
+    bool ok = (lo <= hi) && (hi <= src_bytes) && (len64 <= 4ull * kChunkWindows + 2ull * kChunk) &&
+              (len >= 4u * nwin) && (len <= 4u * nwin + S * nelem) &&
+              (((static_cast<uint32_t>(lo) | len) & 1u) == 0u);
     if (chunk == 0 && lo != 0) ok = false;
     if (chunk == num_chunks - 1 && hi != src_bytes) ok = false;
     if (!ok) {
@@ -356,19 +356,21 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
     uint32_t* t = s_t[warp];
     const uint64_t a0 = lo & ~15ull;
     const uint32_t span = static_cast<uint32_t>(hi - a0);                  // bytes from a0 to the chunk's end
+    // payload bytes behind a0, as far as this chunk can care (32-bit arithmetic in the loop)
+    const uint32_t avail = (src_bytes - a0 > 8192ull) ? 8192u : static_cast<uint32_t>(src_bytes - a0);
+    const uint8_t* from = src + a0;
     for (uint32_t off = 16u * lane; off < span; off += 16u * 32u) {
-        const uint64_t a = a0 + off;
         uint4 q;
         uint32_t nxt = 0;                                                  // the unit behind these 16 bytes
-        if (a + 18 <= src_bytes) {
-            q = __ldcs(reinterpret_cast<const uint4*>(src + a));
-            nxt = *reinterpret_cast<const uint16_t*>(src + a + 16);
+        if (off + 18u <= avail) {
+            q = __ldcs(reinterpret_cast<const uint4*>(from + off));
+            nxt = *reinterpret_cast<const uint16_t*>(from + off + 16);
         } else {
             // the payload's last bytes: never read past src_bytes
             uint32_t wds[4] = {0, 0, 0, 0};
             for (uint32_t b = 0; b < 16; b += 2) {
-                if (a + b + 2 <= src_bytes) {
-                    const uint32_t h = *reinterpret_cast<const uint16_t*>(src + a + b);
+                if (off + b + 2u <= avail) {
+                    const uint32_t h = *reinterpret_cast<const uint16_t*>(from + off + b);
                     wds[b >> 2] |= h << (8 * (b & 2));
                 }
             }
