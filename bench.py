@@ -47,7 +47,7 @@ NOMINAL_HBM_GBS = 8000.0
 # count; writes were below the algorithmic figure because part of the output was
 # still in the write-back L2 at kernel end, a fixed amount that does not scale,
 # so the scaled figure is a slight under-estimate for larger tensors.
-NCU_TRAFFIC_FACTOR = {"zvc_compress_kernel": 0.855, "zvc_decompress_kernel": 0.838}
+NCU_TRAFFIC_FACTOR = {"zvc_compress_kernel": 0.857, "zvc_decompress_kernel": 0.841}
 
 
 def env_int(name, default):
