@@ -253,25 +253,23 @@ struct U16Lane {
 
 // One round = windows 4G .. 4G+3 of a full chunk.  `a` is the shared byte address
 // of the next mask word in t[] minus 8 bytes per window already passed (a mask is
-// two 2-byte units = two 4-byte entries; folded into the immediates).
+// two 2-byte units = two 4-byte entries; folded into the immediates).  The walk is
+// pulled back to the chunk's end after every second window; a walk that was pulled
+// back once overshoots again at every later step, so the caller only looks at `last`.
 template <uint32_t G>
-__device__ __forceinline__ void expand_round_u16(uint32_t& a, uint32_t a_end, bool& bad, const U16Lane& c,
+__device__ __forceinline__ void expand_round_u16(uint32_t& a, uint32_t a_end, uint32_t& last, const U16Lane& c,
                                                  uint2* __restrict__ out) {
     // four serial steps of the self-delimiting walk; every lane sees all four
     const uint32_t a0 = a;
     const uint32_t m0 = lds32<32 * G + 0>(a0);
     const uint32_t a1 = a0 + 4u * __popc(m0);
     const uint32_t m1 = lds32<32 * G + 8>(a1);
-    const uint32_t a2 = a1 + 4u * __popc(m1);
+    const uint32_t a2 = min(a1 + 4u * __popc(m1), a_end - (32u * G + 16u));
     const uint32_t m2 = lds32<32 * G + 16>(a2);
     const uint32_t a3 = a2 + 4u * __popc(m2);
     const uint32_t m3 = lds32<32 * G + 24>(a3);
-    a = a3 + 4u * __popc(m3);
-    // a malformed record may carry the walk past the chunk: flag it and pull the
-    // position back so that no later read leaves the buffer
-    const uint32_t lim = a_end - (32u * G + 32u);
-    bad |= (a > lim);
-    a = min(a, lim);
+    last = a3 + 4u * __popc(m3);
+    a = min(last, a_end - (32u * G + 32u));
     const uint32_t my_a = c.w_hi ? (c.w_odd ? a3 : a2) : (c.w_odd ? a1 : a0);
     const uint32_t my_m = c.w_hi ? (c.w_odd ? m3 : m2) : (c.w_odd ? m1 : m0);
     // the next four values in front of my elements: entries q and q + 2
@@ -282,16 +280,16 @@ __device__ __forceinline__ void expand_round_u16(uint32_t& a, uint32_t a_end, bo
 }
 
 template <uint32_t G>
-__device__ __forceinline__ void expand_rounds_u16(uint32_t& a, uint32_t a_end, bool& bad, const U16Lane& c,
+__device__ __forceinline__ void expand_rounds_u16(uint32_t& a, uint32_t a_end, uint32_t& last, const U16Lane& c,
                                                   uint2* __restrict__ out) {
     if constexpr (G < kChunkWindows / 4) {
-        expand_round_u16<G>(a, a_end, bad, c, out);
-        expand_rounds_u16<G + 1>(a, a_end, bad, c, out);
+        expand_round_u16<G>(a, a_end, last, c, out);
+        expand_rounds_u16<G + 1>(a, a_end, last, c, out);
     }
 }
 
 constexpr uint32_t kU16MaxUnits = 2 * kChunkWindows + kChunk;          // 1088
-constexpr uint32_t kU16Overrun = 4 * (2 + 32);                         // the walk is pulled back every 4 windows
+constexpr uint32_t kU16Overrun = 2 * (2 + 32);                         // the walk is pulled back every 2 windows
 constexpr uint32_t kU16Entries = (kU16MaxUnits + 8 + kU16Overrun + 2 + 36 + 7) / 8 * 8;
 // Expansion table of the 2-byte kernel, indexed by a lane's 4 mask bits:
 // {sel0 | sel1 << 16, keep1}.  Element k takes value number popc(bits below k);
@@ -304,8 +302,8 @@ __constant__ uint2 kExpandU16[16] = {
     {0x32104444u, 0xffffffffu}, {0x54324410u, 0xffffffffu}, {0x54321044u, 0xffffffffu}, {0x76543210u, 0xffffffffu},
 };
 
-// t[] takes 5 KB per warp, so shared memory allows 44 warps per SM: 22 CTAs of 2 warps
-// (small CTAs retire and refill most smoothly; 4 x 11 is 2 % slower, 8 x 5 10 %).
+// t[] takes 4.8 KB per warp, so shared memory allows 46-48 warps per SM; CTAs of 2 warps
+// retire and refill most smoothly (4 warps: 2 % slower, 8 warps: 10 %).
 #ifndef CDMA_DEC16_WARPS
 #define CDMA_DEC16_WARPS 2
 #endif
@@ -413,9 +411,9 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
         c.w_hi = (lane & 16u) != 0u;
         c.w_odd = (lane & 8u) != 0u;
         const uint32_t t_addr = static_cast<uint32_t>(__cvta_generic_to_shared(t));
-        uint32_t a = t_addr + 4u * p;
-        expand_rounds_u16<0>(a, t_addr + 4u * end, bad, c, reinterpret_cast<uint2*>(dst + e0) + lane);
-        p = (a - t_addr) / 4u + kChunkWindows * MU;      // back to units, the 32 mask words included
+        uint32_t a = t_addr + 4u * p, last = 0;
+        expand_rounds_u16<0>(a, t_addr + 4u * end, last, c, reinterpret_cast<uint2*>(dst + e0) + lane);
+        p = (last - t_addr) / 4u + kChunkWindows * MU;   // back to units, the 32 mask words included
     } else {
         // ragged last chunk: lane = element, one window per round
         const uint32_t lt = lanemask_lt();
