@@ -97,8 +97,8 @@ uint64_t cdma_zvc_max_compressed_bytes(uint64_t n, int dtype);
 uint64_t cdma_zvc_table_entries(uint64_t n);
 
 /* Bytes of device scratch a codec call on n elements needs (both directions;
- * a multiple of 256).  Holds the inter-tile prefix descriptors, the tile
- * ticket and the status/result words. */
+ * a multiple of 256).  Holds the status/result words and the inter-tile
+ * prefix descriptors (one per tile of 8192 elements, 32 bytes apart). */
 uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype);
 
 /*
