@@ -222,6 +222,40 @@ int cdma_zvc_decompress_async(const void* d_src, uint64_t src_bytes,
                               uint64_t* h_result);
 
 /* ------------------------------------------------------------------------ *
+ * Run-length comparison codec (Section V-A, "Run-length encoding compression";
+ * its dependence on the activation layout is the subject of Section VI-A,
+ * Fig. 11).  The paper names the scheme but gives no format; this one is the
+ * library's own, on the framing of the zero-value codec: independent chunks of
+ * 1024 elements, a table of cdma_zvc_table_entries(n) byte offsets outside the
+ * payload.  A chunk is a sequence of records {token, literals}: the 32-bit
+ * little-endian token holds the number of zero elements in front (low 16
+ * bits) and the number of non-zero elements that follow (high 16 bits); one
+ * record per maximal run of non-zero elements, plus a last record without
+ * literals when the chunk ends in zeros.  Chunk size = 4 * records + 4 *
+ * non-zero elements, at most 4100 bytes, so cdma_zvc_max_compressed_bytes()
+ * and cdma_zvc_workspace_bytes() size its buffers too.  "Zero" is bitwise.
+ *
+ * dtype must be CDMA_F32 (CDMA_ERR_UNSUPPORTED_DTYPE otherwise).  Arguments,
+ * ownership, alignment, capacity and error behaviour are those of
+ * cdma_zvc_compress / cdma_zvc_decompress and their _async forms; a stream
+ * in which a literal is zero or a token is zero is CDMA_ERR_CORRUPT_STREAM.
+ * ------------------------------------------------------------------------ */
+int64_t cdma_rle_compress(const void* d_src, uint64_t n, int dtype, int layout,
+                          void* d_dst, uint64_t dst_capacity, uint64_t* d_table,
+                          void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
+int cdma_rle_compress_async(const void* d_src, uint64_t n, int dtype, int layout,
+                            void* d_dst, uint64_t dst_capacity, uint64_t* d_table,
+                            void* d_workspace, uint64_t workspace_bytes, void* cuda_stream,
+                            uint64_t* h_result);
+int64_t cdma_rle_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
+                            uint64_t n, int dtype, int layout, void* d_dst,
+                            void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
+int cdma_rle_decompress_async(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
+                              uint64_t n, int dtype, int layout, void* d_dst,
+                              void* d_workspace, uint64_t workspace_bytes, void* cuda_stream,
+                              uint64_t* h_result);
+
+/* ------------------------------------------------------------------------ *
  * Offload pipeline (Section III, Fig. 2b: OFF(n) in the forward pass, PRE(n)
  * in reverse order in the backward pass; Section V-D: the compressed copy
  * replaces the cudaMemcpy calls of the memory manager).

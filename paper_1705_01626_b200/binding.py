@@ -63,6 +63,14 @@ _SIGNATURES = {
                                       c_void_p, c_uint64, c_void_p]),
     "cdma_zvc_decompress_async": (c_int, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p,
                                           c_void_p, c_uint64, c_void_p, c_void_p]),
+    "cdma_rle_compress": (c_int64, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64, c_void_p,
+                                    c_void_p, c_uint64, c_void_p]),
+    "cdma_rle_compress_async": (c_int, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64, c_void_p,
+                                        c_void_p, c_uint64, c_void_p, c_void_p]),
+    "cdma_rle_decompress": (c_int64, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p,
+                                      c_void_p, c_uint64, c_void_p]),
+    "cdma_rle_decompress_async": (c_int, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p,
+                                          c_void_p, c_uint64, c_void_p, c_void_p]),
     "cdma_ctx_create": (c_int, [c_uint64, c_uint64, POINTER(c_void_p)]),
     "cdma_ctx_destroy": (c_int, [c_void_p]),
     "cdma_offload": (c_int64, [c_void_p, c_void_p, c_uint64, c_int, c_int, c_void_p, POINTER(cdma_ticket)]),
@@ -142,6 +150,33 @@ def cdma_zvc_compress_async(d_src, n, dtype, layout, d_dst, dst_capacity, d_tabl
     return int(lib().cdma_zvc_compress_async(_vp(d_src), n, dtype, layout, _vp(d_dst), dst_capacity,
                                              _vp(d_table), _vp(d_workspace), workspace_bytes,
                                              _vp(cuda_stream), _vp(h_result)))
+
+
+def cdma_rle_compress(d_src, n, dtype, layout, d_dst, dst_capacity, d_table, d_workspace,
+                      workspace_bytes, cuda_stream=0) -> int:
+    """Run-length comparison codec (4-byte elements).  Returns the payload size C, or a negative status."""
+    return int(lib().cdma_rle_compress(_vp(d_src), n, dtype, layout, _vp(d_dst), dst_capacity, _vp(d_table),
+                                       _vp(d_workspace), workspace_bytes, _vp(cuda_stream)))
+
+
+def cdma_rle_compress_async(d_src, n, dtype, layout, d_dst, dst_capacity, d_table, d_workspace,
+                            workspace_bytes, cuda_stream, h_result) -> int:
+    return int(lib().cdma_rle_compress_async(_vp(d_src), n, dtype, layout, _vp(d_dst), dst_capacity,
+                                             _vp(d_table), _vp(d_workspace), workspace_bytes,
+                                             _vp(cuda_stream), _vp(h_result)))
+
+
+def cdma_rle_decompress(d_src, src_bytes, d_table, n, dtype, layout, d_dst, d_workspace,
+                        workspace_bytes, cuda_stream=0) -> int:
+    return int(lib().cdma_rle_decompress(_vp(d_src), src_bytes, _vp(d_table), n, dtype, layout, _vp(d_dst),
+                                         _vp(d_workspace), workspace_bytes, _vp(cuda_stream)))
+
+
+def cdma_rle_decompress_async(d_src, src_bytes, d_table, n, dtype, layout, d_dst, d_workspace,
+                              workspace_bytes, cuda_stream, h_result) -> int:
+    return int(lib().cdma_rle_decompress_async(_vp(d_src), src_bytes, _vp(d_table), n, dtype, layout,
+                                               _vp(d_dst), _vp(d_workspace), workspace_bytes,
+                                               _vp(cuda_stream), _vp(h_result)))
 
 
 def cdma_zvc_relu_compress(d_src, n, dtype, layout, d_relu_out, d_dst, dst_capacity, d_table, d_workspace,

@@ -238,6 +238,75 @@ int64_t cdma_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_
     return static_cast<int64_t>(n) * cdma_dtype_size(dtype);
 }
 
+// ---- run-length comparison codec (4-byte elements) -----------------------------------
+
+int cdma_rle_compress_async(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,
+                            uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
+                            uint64_t workspace_bytes, void* cuda_stream, uint64_t* h_result) {
+    const int st = check_common(n, dtype, layout, d_src, d_dst, d_table, d_workspace, workspace_bytes);
+    if (st != CDMA_OK) return st;
+    if (dtype != CDMA_F32) return CDMA_ERR_UNSUPPORTED_DTYPE;
+    if ((dst_capacity != 0 && d_dst == nullptr) || h_result == nullptr) return CDMA_ERR_INVALID_ARG;
+    if (overlaps(d_src, n * 4, d_dst, dst_capacity)) return CDMA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint64_t* ws = static_cast<uint64_t*>(d_workspace);
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * kDescStride * num_tiles_of(n), stream) != cudaSuccess)
+        return CDMA_ERR_CUDA;
+    if (n == 0) {
+        if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    } else if (launch_rle_compress(d_src, n, d_dst, dst_capacity, d_table, ws, stream) != cudaSuccess) {
+        return CDMA_ERR_CUDA;
+    }
+    if (enqueue_result(ws, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    return CDMA_OK;
+}
+
+int64_t cdma_rle_compress(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,
+                          uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
+                          uint64_t workspace_bytes, void* cuda_stream) {
+    uint64_t result[2] = {0, 0};
+    const int st = cdma_rle_compress_async(d_src, n, dtype, layout, d_dst, dst_capacity, d_table, d_workspace,
+                                           workspace_bytes, cuda_stream, result);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (result[1] != 0) return -static_cast<int64_t>(result[1]);
+    return static_cast<int64_t>(result[0]);
+}
+
+int cdma_rle_decompress_async(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                              int dtype, int layout, void* d_dst, void* d_workspace, uint64_t workspace_bytes,
+                              void* cuda_stream, uint64_t* h_result) {
+    const int st = check_common(n, dtype, layout, d_dst, d_src, d_table, d_workspace, workspace_bytes);
+    if (st != CDMA_OK) return st;
+    if (dtype != CDMA_F32) return CDMA_ERR_UNSUPPORTED_DTYPE;
+    if ((src_bytes != 0 && d_src == nullptr) || h_result == nullptr) return CDMA_ERR_INVALID_ARG;
+    if (overlaps(d_dst, n * 4, d_src, src_bytes)) return CDMA_ERR_INVALID_ARG;
+    // sizes the format cannot produce are refused before anything is launched:
+    // at least one token per chunk, at most 1025 words per chunk
+    const uint64_t chunks = num_chunks_of(n);
+    if (src_bytes < 4 * chunks || src_bytes > 4 * (n + chunks) || src_bytes % 4 != 0) return CDMA_ERR_CORRUPT_STREAM;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint64_t* ws = static_cast<uint64_t*>(d_workspace);
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    if (launch_rle_decompress(d_src, src_bytes, d_table, n, d_dst, ws, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    if (enqueue_result(ws, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    return CDMA_OK;
+}
+
+int64_t cdma_rle_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                            int dtype, int layout, void* d_dst, void* d_workspace, uint64_t workspace_bytes,
+                            void* cuda_stream) {
+    uint64_t result[2] = {0, 0};
+    const int st = cdma_rle_decompress_async(d_src, src_bytes, d_table, n, dtype, layout, d_dst, d_workspace,
+                                             workspace_bytes, cuda_stream, result);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (result[1] != 0) return -static_cast<int64_t>(result[1]);
+    return static_cast<int64_t>(n) * 4;
+}
+
 void cdma_time_next_kernel(void* start_event, void* stop_event) {
     t_time_start = static_cast<cudaEvent_t>(start_event);
     t_time_stop = static_cast<cudaEvent_t>(stop_event);

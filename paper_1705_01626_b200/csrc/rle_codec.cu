@@ -1,0 +1,281 @@
+// Run-length comparison codec (Section V-A, "Run-length encoding compression";
+// its layout sensitivity is the subject of Section VI-A, Fig. 11), 4-byte elements.
+//
+// The paper gives no format.  Ours, on the framing of the zero-value codec
+// (independent chunks of 1024 elements, offset table outside the payload): a
+// chunk is a sequence of records {token, literals}; the 32-bit token holds the
+// number of zero elements in front (low 16 bits) and the number of non-zero
+// elements that follow (high 16 bits); a record is written for every maximal run
+// of non-zero elements, and a chunk that ends in zeros gets a last record with
+// no literals.  Chunk size = 4 * records + 4 * non-zero elements.
+//
+// Compression uses the tile / look-back skeleton of the zero-value kernel: one
+// CTA per 8-chunk tile, a warp per chunk, a lane holds one element of each of
+// the chunk's 32 windows, window masks by ballot.  Decompression: a warp per
+// chunk walks the tokens (the walk is serial: a token says where the next one
+// is), builds the dense chunk in shared memory and writes it out once.
+#include "zvc_common.cuh"
+#include "lookback.cuh"
+
+namespace cdma {
+
+namespace {
+
+// r runs need r non-zeros and r - 1 zeros between them, so tokens + literals <= 1025 words per chunk
+constexpr uint32_t kRleMaxChunkUnits = kChunk + 1;
+constexpr uint32_t kBig = 0x7fffffffu;
+
+__global__ void __launch_bounds__(kTileThreads)
+rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
+                    uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
+                    uint64_t num_chunks) {
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    uint32_t* s_tile = reinterpret_cast<uint32_t*>(smem_raw);       // the tile's records, contiguous
+    __shared__ uint32_t s_chunk_units[kTileChunks];
+    __shared__ uint32_t s_next_zero[kTileChunks][kChunkWindows];    // first zero at or after window w + 1
+    __shared__ uint64_t s_base;
+    __shared__ uint32_t s_failed;
+    __shared__ uint32_t s_room;
+
+    const uint32_t lane = lane_id();
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint32_t lt = lanemask_lt();
+    uint64_t* desc = ws + kWsDescriptors;
+    const uint32_t tile = blockIdx.x;          // block-index order, as in the zero-value kernel
+    if (tile >= num_tiles) return;
+
+    // ---- load: lane l takes element l of every window; beyond n: zeros -------------
+    const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunks + warp;
+    const uint64_t e0 = chunk * kChunk;
+    const uint32_t nelem = (e0 >= n) ? 0u : (n - e0 < kChunk ? static_cast<uint32_t>(n - e0) : kChunk);
+    uint32_t e[kChunkWindows];
+#pragma unroll
+    for (uint32_t w = 0; w < kChunkWindows; ++w) {
+        const uint32_t j = w * kWindow + lane;
+        e[w] = (j < nelem) ? __ldcs(src + e0 + j) : 0u;
+    }
+
+    // ---- 1. count: window masks by ballot, lane w keeps the mask of window w --------
+    uint32_t mine = 0;
+#pragma unroll
+    for (uint32_t w = 0; w < kChunkWindows; ++w) {
+        const uint32_t m = __ballot_sync(0xffffffffu, e[w] != 0u);
+        if (lane == w) mine = m;
+    }
+    // lane = window from here: run starts are non-zero elements whose predecessor is zero
+    uint32_t carry = __shfl_up_sync(0xffffffffu, mine >> 31, 1);
+    if (lane == 0) carry = 0;
+    const uint32_t starts = mine & ~((mine << 1) | carry);
+    const uint32_t nnz = __reduce_add_sync(0xffffffffu, __popc(mine));
+    const uint32_t runs = __reduce_add_sync(0xffffffffu, __popc(starts));
+    uint32_t trailing = 0;                                          // the chunk ends in zeros
+    if (nelem != 0) {
+        const uint32_t last_mask = __shfl_sync(0xffffffffu, mine, (nelem - 1) >> 5);
+        trailing = ((last_mask >> ((nelem - 1) & 31u)) & 1u) ^ 1u;
+    }
+    const uint32_t units = runs + trailing + nnz;
+    // first zero at or after each window (suffix minimum), for the run lengths
+    uint32_t fz = (mine != 0xffffffffu) ? lane * kWindow + (__ffs(~mine) - 1) : kBig;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_down_sync(0xffffffffu, fz, o);
+        if (lane + o < 32) fz = min(fz, t);
+    }
+    uint32_t after = __shfl_down_sync(0xffffffffu, fz, 1);          // from window lane + 1 on
+    if (lane == 31) after = kBig;
+    s_next_zero[warp][lane] = min(after, nelem);
+    if (lane == 0) s_chunk_units[warp] = units;
+    __syncthreads();
+    const uint32_t cu = (lane < kTileChunks) ? s_chunk_units[lane] : 0u;
+    const uint32_t chunk_off = __reduce_add_sync(0xffffffffu, lane < warp ? cu : 0u);
+    uint64_t tile_bytes = 0;
+    if (warp == 0) {
+        tile_bytes = static_cast<uint64_t>(__reduce_add_sync(0xffffffffu, cu)) * 4u;
+        if (lane == 0)
+            st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride,
+                           (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+    }
+
+    // ---- 2. assemble the chunk's records in the staged tile --------------------------
+    uint32_t* st = s_tile + chunk_off;
+    uint32_t nnz_run = 0, runs_run = 0;          // non-zeros and run starts in front of this window
+    int32_t last_nz = -1;                        // index of the last non-zero element in front of it
+    uint32_t prev_top = 0;                       // bit 31 of the previous window's mask
+#pragma unroll
+    for (uint32_t w = 0; w < kChunkWindows; ++w) {
+        const uint32_t m = __ballot_sync(0xffffffffu, e[w] != 0u);
+        const uint32_t sw = m & ~((m << 1) | prev_top);
+        const uint32_t i = w * kWindow + lane;                      // my element's index in the chunk
+        // my place: one word per record started up to and including me, one per non-zero before me
+        const uint32_t pos = runs_run + __popc(sw & (lt | (1u << lane))) + nnz_run + __popc(m & lt);
+        if ((m >> lane) & 1u) st[pos] = e[w];
+        if ((sw >> lane) & 1u) {
+            const uint32_t lower = m & lt;
+            const uint32_t zeros = lower ? (lane - 1u - (31u - __clz(lower)))
+                                         : static_cast<uint32_t>(static_cast<int32_t>(i) - 1 - last_nz);
+            const uint32_t higher_zeros = ~m & ~(lt | (1u << lane));
+            const uint32_t run_end = higher_zeros ? w * kWindow + (__ffs(higher_zeros) - 1) : s_next_zero[warp][w];
+            st[pos - 1] = zeros | ((run_end - i) << 16);
+        }
+        nnz_run += __popc(m);
+        runs_run += __popc(sw);
+        if (m) last_nz = static_cast<int32_t>(w * kWindow + 31u - __clz(m));
+        prev_top = m >> 31;
+    }
+    if (trailing && lane == 0) st[units - 1] = nelem - 1u - static_cast<uint32_t>(last_nz);   // zeros only
+
+    // ---- 3. the tile's place in the stream ------------------------------------------
+    if (warp == 0) {
+        LookbackResult lb{0, false};
+        if (tile != 0) {
+            lb = lookback_walk(desc, ws, tile);
+            if (lane == 0)
+                st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride,
+                               lb.failed ? kDescError : (kDescPrefix | (lb.exclusive + tile_bytes)));
+        }
+        if (lane == 0) {
+            s_base = lb.exclusive;
+            s_failed = lb.failed ? 1u : 0u;
+            const uint64_t end_bytes = lb.exclusive + tile_bytes;
+            s_room = static_cast<uint32_t>((cap >= end_bytes ? tile_bytes : (cap > lb.exclusive ? cap - lb.exclusive : 0)) / 4u);
+            if (!lb.failed) {
+                if (tile == num_tiles - 1) {
+                    table[num_chunks] = end_bytes;
+                    ws[kWsBytes] = end_bytes;
+                }
+                if (end_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
+            }
+        }
+    }
+    __syncthreads();
+    if (s_failed) return;
+
+    // ---- 4. the CTA writes the tile's words to their place, below cap ----------------
+    const uint64_t first_unit = s_base / 4u;
+    if (lane == 0 && chunk < num_chunks) table[chunk] = (first_unit + chunk_off) * 4u;
+    const uint32_t room = s_room;
+    uint32_t* out = reinterpret_cast<uint32_t*>(dst) + first_unit;
+    for (uint32_t u = threadIdx.x; u < room; u += kTileThreads) out[u] = s_tile[u];
+}
+
+constexpr uint32_t kRleDecWarps = 4;
+
+__global__ void __launch_bounds__(32 * kRleDecWarps)
+rle_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const uint64_t* __restrict__ table,
+                      uint64_t n, uint32_t* __restrict__ dst, uint64_t* __restrict__ ws, uint64_t num_chunks) {
+    // staged payload (16-byte phase in front) and the dense chunk being built
+    constexpr uint32_t kStageWords = kRleMaxChunkUnits + 4 + 3;
+    __shared__ __align__(16) uint32_t s_stage[kRleDecWarps][(kStageWords + 3) / 4 * 4];
+    __shared__ __align__(16) uint32_t s_dense[kRleDecWarps][kChunk];
+
+    const uint32_t lane = lane_id();
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * kRleDecWarps + warp;
+    if (blockIdx.x == 0 && threadIdx.x == 0) ws[kWsBytes] = n * 4u;
+    if (chunk >= num_chunks) return;
+    const uint64_t e0 = chunk * kChunk;
+    const uint32_t nelem = (n - e0 < kChunk) ? static_cast<uint32_t>(n - e0) : kChunk;
+
+    // ---- the chunk's byte range, validated ---------------------------------------------
+    const uint64_t lo = __ldg(table + chunk);
+    const uint64_t hi = __ldg(table + chunk + 1);
+    const uint64_t len64 = hi - lo;
+    bool ok = (lo <= hi) && (hi <= src_bytes) && (len64 >= 4) && (len64 <= 4ull * kRleMaxChunkUnits) &&
+              (((static_cast<uint32_t>(lo) | static_cast<uint32_t>(len64)) & 3u) == 0u);
+    if (chunk == 0 && lo != 0) ok = false;
+    if (chunk == num_chunks - 1 && hi != src_bytes) ok = false;
+    if (!ok) {
+        if (lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+        return;
+    }
+
+    // ---- stage payload bytes [lo, hi); zero the dense chunk -----------------------------
+    uint32_t* buf = s_stage[warp];
+    uint32_t* dense = s_dense[warp];
+    const uint64_t a0 = lo & ~15ull;
+    const uint32_t span = static_cast<uint32_t>(hi - a0);
+    for (uint32_t off = 16u * lane; off < span; off += 16u * 32u) {
+        uint4 q = make_uint4(0, 0, 0, 0);
+        if (a0 + off + 16 <= src_bytes) {
+            q = __ldcs(reinterpret_cast<const uint4*>(src + a0 + off));
+        } else {
+            uint32_t wds[4] = {0, 0, 0, 0};
+            for (uint32_t b = 0; b < 16; b += 4)
+                if (a0 + off + b + 4 <= src_bytes) wds[b >> 2] = *reinterpret_cast<const uint32_t*>(src + a0 + off + b);
+            q = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+        }
+        *reinterpret_cast<uint4*>(buf + off / 4) = q;
+    }
+#pragma unroll
+    for (uint32_t k = 0; k < kChunk / 128; ++k) reinterpret_cast<uint4*>(dense)[k * 32 + lane] = make_uint4(0, 0, 0, 0);
+    __syncwarp();
+
+    // ---- walk the records: every lane sees every token; lanes share a record's literals ----
+    uint32_t p = static_cast<uint32_t>(lo - a0) / 4u;
+    const uint32_t end = span / 4u;
+    uint32_t pos = 0;
+    bool bad = false;
+    while (pos < nelem) {
+        if (p >= end) { bad = true; break; }
+        const uint32_t token = buf[p];
+        const uint32_t zeros = token & 0xffffu, count = token >> 16;
+        if (token == 0u || pos + zeros + count > nelem || p + 1 + count > end) { bad = true; break; }
+        for (uint32_t j = lane; j < count; j += 32) {
+            const uint32_t v = buf[p + 1 + j];
+            bad |= (v == 0u);
+            dense[pos + zeros + j] = v;
+        }
+        p += 1 + count;
+        pos += zeros + count;
+    }
+    bad = __any_sync(0xffffffffu, bad) || p != end;
+    __syncwarp();
+    if (bad) {
+        if (lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+        return;
+    }
+
+    // ---- write the dense chunk once -------------------------------------------------------
+    if (nelem == kChunk) {
+        uint4* out = reinterpret_cast<uint4*>(dst + e0);
+#pragma unroll
+        for (uint32_t k = 0; k < kChunk / 128; ++k) __stcs(out + k * 32 + lane, reinterpret_cast<const uint4*>(dense)[k * 32 + lane]);
+    } else {
+        for (uint32_t j = lane; j < nelem; j += 32) dst[e0 + j] = dense[j];
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_rle_compress(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
+                                uint64_t* d_ws, cudaStream_t stream) {
+    const uint64_t chunks = num_chunks_of(n);
+    const uint64_t tiles = num_tiles_of(n);
+    if (tiles == 0) return cudaSuccess;
+    constexpr uint32_t kSmem = kTileChunks * kRleMaxChunkUnits * 4;
+    const cudaError_t e = cudaFuncSetAttribute(rle_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    timing_before_launch(stream);
+    rle_compress_kernel<<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
+        static_cast<const uint32_t*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
+        static_cast<uint32_t>(tiles), chunks);
+    timing_after_launch(stream);
+    count_kernel_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rle_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                  void* d_dst, uint64_t* d_ws, cudaStream_t stream) {
+    const uint64_t chunks = num_chunks_of(n);
+    if (chunks == 0) return cudaSuccess;
+    const dim3 grid(static_cast<unsigned>((chunks + kRleDecWarps - 1) / kRleDecWarps));
+    timing_before_launch(stream);
+    rle_decompress_kernel<<<grid, 32 * kRleDecWarps, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes,
+                                                                   d_table, n, static_cast<uint32_t*>(d_dst), d_ws,
+                                                                   chunks);
+    timing_after_launch(stream);
+    count_kernel_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace cdma

@@ -95,6 +95,10 @@ cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t ele
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
                                   cudaStream_t stream, bool src_on_device = true);
+cudaError_t launch_rle_compress(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
+                                uint64_t* d_ws, cudaStream_t stream);
+cudaError_t launch_rle_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                  void* d_dst, uint64_t* d_ws, cudaStream_t stream);
 void count_kernel_launch();
 void timing_before_launch(cudaStream_t stream);   // measurement hook, see cdma_time_next_kernel
 void timing_after_launch(cudaStream_t stream);
