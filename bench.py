@@ -550,8 +550,13 @@ def run_e2e(B, x, code, c_bytes, args, world, dev):
 # --------------------------------------------------------------------------- #
 # results-table workloads (not the default line): offload set and layout sweep
 # --------------------------------------------------------------------------- #
-def time_codec(B, x, code, iters=10):
-    """Device-timed compress and decompress of one tensor: (C, ms_compress, ms_decompress)."""
+def time_codec(B, x, code, iters=10, codec="zvc"):
+    """Device-timed compress and decompress of one tensor: (C, ms_compress, ms_decompress).
+    codec: "zvc" (the paper's zero-value compression) or "rle" (the run-length comparison codec)."""
+    comp, comp_async = (B.cdma_zvc_compress, B.cdma_zvc_compress_async) if codec == "zvc" else \
+        (B.cdma_rle_compress, B.cdma_rle_compress_async)
+    dec, dec_async = (B.cdma_zvc_decompress, B.cdma_zvc_decompress_async) if codec == "zvc" else \
+        (B.cdma_rle_decompress, B.cdma_rle_decompress_async)
     import torch
     n = x.numel()
     cap = B.cdma_zvc_max_compressed_bytes(n, code)
@@ -563,11 +568,11 @@ def time_codec(B, x, code, iters=10):
     out = torch.empty_like(x)
     res = torch.zeros(2, dtype=torch.int64).pin_memory()
     sh = torch.cuda.current_stream().cuda_stream
-    c = B.cdma_zvc_compress(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
+    c = comp(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
                             ws.data_ptr(), ws_bytes, sh)
     if c < 0:
-        raise B.CdmaError(c, "cdma_zvc_compress")
-    r = B.cdma_zvc_decompress(payload.data_ptr(), c, table.data_ptr(), n, code, B.NCHW, out.data_ptr(),
+        raise B.CdmaError(c, "compress")
+    r = dec(payload.data_ptr(), c, table.data_ptr(), n, code, B.NCHW, out.data_ptr(),
                               ws.data_ptr(), ws_bytes, sh)
     it = torch.int32 if x.element_size() == 4 else torch.int16
     if r < 0 or not torch.equal(out.view(-1).view(it), x.view(-1).view(it)):
@@ -579,13 +584,13 @@ def time_codec(B, x, code, iters=10):
         flush.fill_(i & 0xFF)                      # tensors smaller than L2 are measured cold
         a, b, cc = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         a.record()
-        B.cdma_zvc_compress_async(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
+        comp_async(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
                                   ws.data_ptr(), ws_bytes, sh, res.data_ptr())
         b.record()
         flush.fill_((i + 1) & 0xFF)
         d0 = torch.cuda.Event(enable_timing=True)
         d0.record()
-        B.cdma_zvc_decompress_async(payload.data_ptr(), c, table.data_ptr(), n, code, B.NCHW, out.data_ptr(),
+        dec_async(payload.data_ptr(), c, table.data_ptr(), n, code, B.NCHW, out.data_ptr(),
                                     ws.data_ptr(), ws_bytes, sh, res.data_ptr())
         cc.record()
         torch.cuda.synchronize()
@@ -596,7 +601,9 @@ def time_codec(B, x, code, iters=10):
 
 
 def run_sweep(args):
-    """config4: ratio and GB/s per (density, layout); tensors (103 MB) are measured with a cold L2."""
+    """config4: ratio and GB/s per (density, layout); tensors (103 MB) are measured with a cold L2.
+    Each point also goes through the run-length comparison codec (Section VI-A, Fig. 11: zero-value
+    compression gives the same ratio in every layout, run-length encoding does not)."""
     import torch
     from paper_1705_01626_b200 import binding as B
     from paper_1705_01626_b200 import workloads as wl
@@ -604,13 +611,20 @@ def run_sweep(args):
     peak, kind = measured_peak()
     for d, layout, x in wl.layout_density_sweep(device="cuda"):
         c, tc, td = time_codec(B, x, B.F32)
+        rc, rtc, rtd = time_codec(B, x, B.F32, codec="rle")
         dense = x.numel() * 4
         algo = dense + c + 8 * B.cdma_zvc_table_entries(x.numel())
+        ralgo = dense + rc + 8 * B.cdma_zvc_table_entries(x.numel())
         print(json.dumps({"workload": "config4", "density": d, "layout": layout, "dense_bytes": dense,
                           "compressed_bytes": c, "ratio": dense / c,
                           "compress_GBps": dense / tc / 1e6, "decompress_GBps": dense / td / 1e6,
                           "compress_frac_of_" + kind: algo / tc / 1e6 / peak,
-                          "decompress_frac_of_" + kind: algo / td / 1e6 / peak, "l2": "flushed between calls"}),
+                          "decompress_frac_of_" + kind: algo / td / 1e6 / peak,
+                          "rle": {"compressed_bytes": rc, "ratio": dense / rc,
+                                  "compress_GBps": dense / rtc / 1e6, "decompress_GBps": dense / rtd / 1e6,
+                                  "compress_frac_of_" + kind: ralgo / rtc / 1e6 / peak,
+                                  "decompress_frac_of_" + kind: ralgo / rtd / 1e6 / peak},
+                          "l2": "flushed between calls"}),
               flush=True)
 
 

@@ -1,7 +1,12 @@
 """Plain numpy statement of the run-length comparison codec (Section V-A,
 "Run-length encoding compression").
 
-TEST INFRASTRUCTURE -- see the package docstring.  The paper names run-length
+TEST INFRASTRUCTURE -- see the package docstring.  PARITY UNPINNED against the
+paper: it prints no format and no worked example for this scheme, so this file
+is pinned only by hand-worked streams of the format stated below, the size
+formula against brute-force run counting, round trips and invariants.
+
+The paper names run-length
 encoding as the first scheme it tried and reports how its ratio depends on the
 activation layout (Section VI-A, Fig. 11), but gives no format.  The format
 below is this build's own (stated in the design document); what the paper fixes

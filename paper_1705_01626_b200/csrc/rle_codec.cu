@@ -13,7 +13,8 @@
 // CTA per 8-chunk tile, a warp per chunk, a lane holds one element of each of
 // the chunk's 32 windows, window masks by ballot.  Decompression: a warp per
 // chunk walks the tokens (the walk is serial: a token says where the next one
-// is), builds the dense chunk in shared memory and writes it out once.
+// is), zero-fills its chunk of the output and stores each record's literals over
+// the zeros (never outside the chunk, whatever the stream holds).
 #include "zvc_common.cuh"
 #include "lookback.cuh"
 
@@ -25,7 +26,7 @@ namespace {
 constexpr uint32_t kRleMaxChunkUnits = kChunk + 1;
 constexpr uint32_t kBig = 0x7fffffffu;
 
-__global__ void __launch_bounds__(kTileThreads)
+__global__ void __launch_bounds__(kTileThreads, 4)
 rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
                     uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
                     uint64_t num_chunks) {
@@ -108,15 +109,17 @@ rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __res
         const uint32_t i = w * kWindow + lane;                      // my element's index in the chunk
         // my place: one word per record started up to and including me, one per non-zero before me
         const uint32_t pos = runs_run + __popc(sw & (lt | (1u << lane))) + nnz_run + __popc(m & lt);
-        if ((m >> lane) & 1u) st[pos] = e[w];
-        if ((sw >> lane) & 1u) {
-            const uint32_t lower = m & lt;
-            const uint32_t zeros = lower ? (lane - 1u - (31u - __clz(lower)))
-                                         : static_cast<uint32_t>(static_cast<int32_t>(i) - 1 - last_nz);
-            const uint32_t higher_zeros = ~m & ~(lt | (1u << lane));
-            const uint32_t run_end = higher_zeros ? w * kWindow + (__ffs(higher_zeros) - 1) : s_next_zero[warp][w];
-            st[pos - 1] = zeros | ((run_end - i) << 16);
-        }
+        // (no branch: every lane works out the token its element would start; only run starts store it)
+        const uint32_t lower = m & lt;
+        const uint32_t zeros = lower ? (lane - 1u - (31u - __clz(lower)))
+                                     : static_cast<uint32_t>(static_cast<int32_t>(i) - 1 - last_nz);
+        const uint32_t higher_zeros = ~m & ~(lt | (1u << lane));
+        const uint32_t beyond = s_next_zero[warp][w];
+        const uint32_t run_end = higher_zeros ? w * kWindow + (__ffs(higher_zeros) - 1) : beyond;
+        const uint32_t s_addr = static_cast<uint32_t>(__cvta_generic_to_shared(st + pos));
+        asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t@p st.shared.u32 [%0], %1;\n\t"
+                     "setp.ne.u32 q, %3, 0;\n\t@q st.shared.u32 [%0+-4], %2;\n\t}"
+                     ::"r"(s_addr), "r"(e[w]), "r"(zeros | ((run_end - i) << 16)), "r"((sw >> lane) & 1u) : "memory");
         nnz_run += __popc(m);
         runs_run += __popc(sw);
         if (m) last_nz = static_cast<int32_t>(w * kWindow + 31u - __clz(m));
@@ -158,15 +161,14 @@ rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __res
     for (uint32_t u = threadIdx.x; u < room; u += kTileThreads) out[u] = s_tile[u];
 }
 
-constexpr uint32_t kRleDecWarps = 4;
+constexpr uint32_t kRleDecWarps = 8;
 
 __global__ void __launch_bounds__(32 * kRleDecWarps)
 rle_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const uint64_t* __restrict__ table,
                       uint64_t n, uint32_t* __restrict__ dst, uint64_t* __restrict__ ws, uint64_t num_chunks) {
-    // staged payload (16-byte phase in front) and the dense chunk being built
+    // staged payload (16-byte phase in front)
     constexpr uint32_t kStageWords = kRleMaxChunkUnits + 4 + 3;
     __shared__ __align__(16) uint32_t s_stage[kRleDecWarps][(kStageWords + 3) / 4 * 4];
-    __shared__ __align__(16) uint32_t s_dense[kRleDecWarps][kChunk];
 
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
@@ -191,7 +193,7 @@ rle_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const
 
     // ---- stage payload bytes [lo, hi); zero the dense chunk -----------------------------
     uint32_t* buf = s_stage[warp];
-    uint32_t* dense = s_dense[warp];
+    uint32_t* dense = dst + e0;                  // zero-filled first, literals stored over the zeros
     const uint64_t a0 = lo & ~15ull;
     const uint32_t span = static_cast<uint32_t>(hi - a0);
     for (uint32_t off = 16u * lane; off < span; off += 16u * 32u) {
@@ -206,43 +208,45 @@ rle_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const
         }
         *reinterpret_cast<uint4*>(buf + off / 4) = q;
     }
+    if (nelem == kChunk) {
 #pragma unroll
-    for (uint32_t k = 0; k < kChunk / 128; ++k) reinterpret_cast<uint4*>(dense)[k * 32 + lane] = make_uint4(0, 0, 0, 0);
-    __syncwarp();
+        for (uint32_t k = 0; k < kChunk / 128; ++k) reinterpret_cast<uint4*>(dense)[k * 32 + lane] = make_uint4(0, 0, 0, 0);
+    } else {
+        for (uint32_t j = lane; j < nelem; j += 32) dense[j] = 0u;
+    }
+    __syncwarp();                                // the zeros are ordered before this warp's literal stores
 
     // ---- walk the records: every lane sees every token; lanes share a record's literals ----
     uint32_t p = static_cast<uint32_t>(lo - a0) / 4u;
     const uint32_t end = span / 4u;
     uint32_t pos = 0;
     bool bad = false;
+    uint32_t zero_literal = 0;                   // per lane: a literal that is zero was seen
     while (pos < nelem) {
-        if (p >= end) { bad = true; break; }
-        const uint32_t token = buf[p];
+        // (reading one word past `end` is harmless: the staging buffer has room and the
+        // checks below refuse whatever it holds)
+        const uint32_t token = buf[min(p, end)];
         const uint32_t zeros = token & 0xffffu, count = token >> 16;
-        if (token == 0u || pos + zeros + count > nelem || p + 1 + count > end) { bad = true; break; }
-        for (uint32_t j = lane; j < count; j += 32) {
-            const uint32_t v = buf[p + 1 + j];
-            bad |= (v == 0u);
-            dense[pos + zeros + j] = v;
+        if (p >= end || token == 0u || pos + zeros + count > nelem || p + 1 + count > end) { bad = true; break; }
+        const uint32_t from = p + 1 + lane, to = pos + zeros + lane;
+        if (lane < count) {                      // runs of up to 32 literals: one step
+            const uint32_t v = buf[from];
+            zero_literal |= (v == 0u) ? 1u : 0u;
+            dense[to] = v;
+        }
+        for (uint32_t j = 32; j < count; j += 32) {
+            if (lane + j < count) {
+                const uint32_t v = buf[from + j];
+                zero_literal |= (v == 0u) ? 1u : 0u;
+                dense[to + j] = v;
+            }
         }
         p += 1 + count;
         pos += zeros + count;
     }
+    bad |= zero_literal != 0u;
     bad = __any_sync(0xffffffffu, bad) || p != end;
-    __syncwarp();
-    if (bad) {
-        if (lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
-        return;
-    }
-
-    // ---- write the dense chunk once -------------------------------------------------------
-    if (nelem == kChunk) {
-        uint4* out = reinterpret_cast<uint4*>(dst + e0);
-#pragma unroll
-        for (uint32_t k = 0; k < kChunk / 128; ++k) __stcs(out + k * 32 + lane, reinterpret_cast<const uint4*>(dense)[k * 32 + lane]);
-    } else {
-        for (uint32_t j = lane; j < nelem; j += 32) dst[e0 + j] = dense[j];
-    }
+    if (bad && lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
 }
 
 }  // namespace
