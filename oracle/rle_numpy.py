@@ -9,7 +9,7 @@ formula against brute-force run counting, round trips and invariants.
 The paper names run-length
 encoding as the first scheme it tried and reports how its ratio depends on the
 activation layout (Section VI-A, Fig. 11), but gives no format.  The format
-below is this build's own (stated in the design document); what the paper fixes
+below is this build's own; what the paper fixes
 is only the idea: runs of zeros are replaced by their length, so the scheme
 pays off for consecutive zeros and is sensitive to the memory layout.
 

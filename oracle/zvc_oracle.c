@@ -22,7 +22,7 @@
  *     population count of a mask tells how many values follow it, the
  *     position of the next mask is known from the stream alone.
  *
- * Readings where the paper is silent (all listed in the design document):
+ * Readings where the paper is silent:
  * bit i (least significant = 0) belongs to element i of the window; the mask
  * is stored least-significant byte first; a short last window has zero bits
  * for the missing elements and no values for them; for 2-byte elements the
