@@ -123,8 +123,12 @@ uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype);
  * table = {0}.
  *
  * cdma_zvc_compress_async only enqueues.  h_result must point to two uint64
- * in pinned host memory; once the stream reaches that point h_result[0] holds
- * C and h_result[1] the status code (0 on success).
+ * in host memory, 8-byte aligned; once the stream reaches that point
+ * h_result[0] holds C and h_result[1] the status code (0 on success).  With
+ * page-locked memory (recommended) the two words are stored by a one-warp
+ * kernel behind the codec kernel; pageable memory gets a 16-byte copy instead.
+ * d_src, d_dst and d_table may also be device views of page-locked host
+ * memory: the kernel then reads / writes over the host link directly.
  */
 int64_t cdma_zvc_compress(const void* d_src, uint64_t n, int dtype, int layout,
                           void* d_dst, uint64_t dst_capacity, uint64_t* d_table,
