@@ -296,6 +296,27 @@ int64_t cdma_offload(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, in
                      void* compute_stream, cdma_ticket* out);
 
 /*
+ * OFF without a host-side wait (Fig. 2b: the offload of layer n's map runs beside
+ * the forward computation of the layers that follow; Section V-D: the compressed
+ * size is reported on completion).  The call enqueues the compression on
+ * compute_stream and, behind it on the context's side stream, a small copy kernel
+ * that reads the payload size on the device and stores exactly that many bytes,
+ * plus the table, into the (mapped) pinned pool; it returns a ticket at once,
+ * without waiting for anything the caller has enqueued on compute_stream.
+ * Returns a status.  The pinned pool holds a worst-case reservation for the
+ * ticket until its size is first needed -- by cdma_ticket_info,
+ * cdma_ticket_host_view, cdma_prefetch*, cdma_ctx_synchronize or a later
+ * reservation that does not fit -- which waits for the ticket's bytes to have
+ * landed and gives the unused part back.  A failure of the compression (for
+ * instance a staging slot too small for the payload) drops the ticket and is
+ * reported by cdma_ctx_synchronize; the ticket is then unknown.  d_src must stay
+ * unchanged until the compression kernel has run (stream order on
+ * compute_stream guarantees it for work enqueued later on that stream).
+ */
+int cdma_offload_async(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, int layout,
+                       void* compute_stream, cdma_ticket* out);
+
+/*
  * PRE: enqueue the host-to-device copy of the ticket's payload and table on
  * the side stream, then the decompression into d_dst on compute_stream once
  * the copy has landed.  The ticket and its pinned bytes are released.

@@ -74,6 +74,7 @@ _SIGNATURES = {
     "cdma_ctx_create": (c_int, [c_uint64, c_uint64, POINTER(c_void_p)]),
     "cdma_ctx_destroy": (c_int, [c_void_p]),
     "cdma_offload": (c_int64, [c_void_p, c_void_p, c_uint64, c_int, c_int, c_void_p, POINTER(cdma_ticket)]),
+    "cdma_offload_async": (c_int, [c_void_p, c_void_p, c_uint64, c_int, c_int, c_void_p, POINTER(cdma_ticket)]),
     "cdma_prefetch": (c_int64, [c_void_p, cdma_ticket, c_void_p, c_void_p]),
     "cdma_prefetch_async": (c_int, [c_void_p, cdma_ticket, c_void_p, c_void_p]),
     "cdma_offload_direct": (c_int64, [c_void_p, c_void_p, c_uint64, c_int, c_int, c_void_p, POINTER(cdma_ticket)]),
@@ -235,6 +236,13 @@ def cdma_offload(ctx, d_src, n, dtype, layout, compute_stream=0):
     t = cdma_ticket(0)
     r = lib().cdma_offload(ctx, _vp(d_src), n, dtype, layout, _vp(compute_stream), ctypes.byref(t))
     return int(r), t
+
+
+def cdma_offload_async(ctx, d_src, n, dtype, layout, compute_stream=0):
+    """Enqueue compression and the copy to the pinned pool without waiting.  Returns (status, ticket)."""
+    t = cdma_ticket(0)
+    st = lib().cdma_offload_async(ctx, _vp(d_src), n, dtype, layout, _vp(compute_stream), ctypes.byref(t))
+    return int(st), t
 
 
 def cdma_prefetch(ctx, ticket, d_dst, compute_stream=0) -> int:

@@ -1,7 +1,12 @@
-// extern "C" codec entry points: argument checking, workspace reset, launch,
-// result read-back.  Declarations and contracts are in include/cdma.h.
+// extern "C" codec entry points: argument checking, launch, result hand-over.
+// Declarations and contracts are in include/cdma.h.
 #include <atomic>
+#include <chrono>
 #include <cstring>
+#include <mutex>
+#include <random>
+#include <utility>
+#include <vector>
 
 #include "zvc_common.cuh"
 
@@ -24,34 +29,73 @@ void timing_after_launch(cudaStream_t stream) {
     t_time_stop = nullptr;
 }
 
-// Result words of a launch, handed to the host.  Page-locked host memory is
-// addressable from the device, so a one-warp kernel stores the two words there
-// (the next thing on the stream, with no copy-engine hand-over, which costs about
-// 10 us per call); any other destination takes an ordinary 16-byte copy.
-__global__ void publish_result_kernel(const uint64_t* __restrict__ ws, uint64_t* __restrict__ out) {
-    if (threadIdx.x < 2) out[threadIdx.x] = ws[kWsBytes + threadIdx.x];
-}
-
-static cudaError_t enqueue_result(const uint64_t* ws, uint64_t* h_result, cudaStream_t stream) {
-    cudaPointerAttributes attr;
-    if (cudaPointerGetAttributes(&attr, h_result) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
-        attr.devicePointer != nullptr && aligned_u64(attr.devicePointer)) {
-        publish_result_kernel<<<1, 32, 0, stream>>>(ws, static_cast<uint64_t*>(attr.devicePointer));
-        count_kernel_launch();
-        return cudaGetLastError();
+// Tags of launches: a process-wide counter started at a value that differs from
+// run to run, so that a workspace written by another process (or left dirty by the
+// caller) does not hold a matching tag either.
+static std::atomic<uint64_t> g_next_tag{0};
+static uint64_t fresh_tag() {
+    uint64_t t = g_next_tag.load(std::memory_order_relaxed);
+    if (t == 0) {
+        const uint64_t seed = (static_cast<uint64_t>(std::chrono::steady_clock::now().time_since_epoch().count()) *
+                               0x9E3779B97F4A7C15ull) ^ (static_cast<uint64_t>(std::random_device{}()) << 20);
+        uint64_t expected = 0;
+        g_next_tag.compare_exchange_strong(expected, (seed & kTagMask) | 1ull);
     }
-    (void)cudaGetLastError();   // an unregistered pointer is not an error here
-    return cudaMemcpyAsync(h_result, ws + kWsBytes, 16, cudaMemcpyDeviceToHost, stream);
+    do {
+        t = g_next_tag.fetch_add(1, std::memory_order_relaxed) & kTagMask;
+    } while (t == 0);
+    return t;
 }
 
 // True when p lies in page-locked host memory (which kernels reach over the host link).
-static bool in_host_memory(const void* p) {
+bool in_host_memory(const void* p) {
     cudaPointerAttributes attr;
     if (p == nullptr || cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
         (void)cudaGetLastError();
         return false;
     }
     return attr.type == cudaMemoryTypeHost;
+}
+
+// Page-locked host memory is addressable from the device, so the kernel that knows
+// the result stores the two words there itself: no extra operation on the stream.
+LaunchCtl make_launch_ctl(uint64_t* h_result) {
+    LaunchCtl ctl{fresh_tag(), nullptr, kWaitLimitNs, kNoTile};
+    cudaPointerAttributes attr;
+    if (h_result != nullptr && cudaPointerGetAttributes(&attr, h_result) == cudaSuccess &&
+        attr.type == cudaMemoryTypeHost && attr.devicePointer != nullptr && aligned_u64(attr.devicePointer))
+        ctl.result_out = static_cast<uint64_t*>(attr.devicePointer);
+    else
+        (void)cudaGetLastError();   // an unregistered pointer is not an error here
+    return ctl;
+}
+
+// Any other destination takes an ordinary 16-byte copy behind the kernel.
+cudaError_t finish_result(const uint64_t* d_ws, const LaunchCtl& ctl, uint64_t* h_result, cudaStream_t stream) {
+    if (ctl.result_out != nullptr) return cudaSuccess;
+    return cudaMemcpyAsync(h_result, d_ws + kWsBytes, 16, cudaMemcpyDeviceToHost, stream);
+}
+
+cudaError_t result_without_kernel(uint64_t* d_ws, uint64_t bytes, uint64_t* h_result, cudaStream_t stream) {
+    // only n = 0 comes here, where bytes is 0 too: both words are zero
+    (void)bytes;
+    const cudaError_t e = cudaMemsetAsync(d_ws + kWsBytes, 0, 16, stream);
+    if (e != cudaSuccess) return e;
+    return cudaMemcpyAsync(h_result, d_ws + kWsBytes, 16, cudaMemcpyDeviceToHost, stream);
+}
+
+cudaError_t opt_in_shared_memory(const void* kernel, uint32_t bytes) {
+    static std::mutex mu;
+    static std::vector<std::pair<const void*, int>> done;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const auto& d : done)
+        if (d.first == kernel && d.second == dev) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    if (e == cudaSuccess) done.emplace_back(kernel, dev);
+    return e;
 }
 
 static inline bool aligned(const void* p, uintptr_t a) {
@@ -124,6 +168,27 @@ uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype) {
     return (bytes + 255) & ~255ull;
 }
 
+// Launch and result hand-over shared by every compression entry point.
+static int compress_launch(const void* d_src, uint64_t n, int dtype, bool relu, void* d_relu_out, void* d_dst,
+                           uint64_t dst_capacity, uint64_t* d_table, uint64_t* ws, const LaunchCtl& ctl,
+                           cudaStream_t stream, uint64_t* h_result) {
+    const uint32_t s = cdma_dtype_size(dtype);
+    if (n == 0) {
+        if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+        if (result_without_kernel(ws, 0, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+        return CDMA_OK;
+    }
+    const bool on_device = !in_host_memory(d_src);
+    const uint32_t nan_above = (dtype == CDMA_F32) ? 0x7f800000u : (dtype == CDMA_F16 ? 0x7c00u : 0x7f80u);
+    const cudaError_t e =
+        relu ? launch_zvc_relu_compress(d_src, n, s, nan_above, d_relu_out, d_dst, dst_capacity, d_table, ws, ctl,
+                                        stream, on_device)
+             : launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, ctl, stream, on_device);
+    if (e != cudaSuccess) return CDMA_ERR_CUDA;
+    if (finish_result(ws, ctl, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    return CDMA_OK;
+}
+
 // Shared body of the plain and the ReLU-fused compression calls.
 static int compress_enqueue(const void* d_src, uint64_t n, int dtype, int layout, bool relu, void* d_relu_out,
                             void* d_dst, uint64_t dst_capacity, uint64_t* d_table, void* d_workspace,
@@ -143,22 +208,8 @@ static int compress_enqueue(const void* d_src, uint64_t n, int dtype, int layout
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint64_t* ws = static_cast<uint64_t*>(d_workspace);
 
-    // result words and every tile descriptor start at zero
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * kDescStride * num_tiles_of(n), stream) != cudaSuccess)
-        return CDMA_ERR_CUDA;
-    if (n == 0) {
-        if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return CDMA_ERR_CUDA;
-    } else {
-        const bool on_device = !in_host_memory(d_src);
-        const uint32_t nan_above = (dtype == CDMA_F32) ? 0x7f800000u : (dtype == CDMA_F16 ? 0x7c00u : 0x7f80u);
-        const cudaError_t e =
-            relu ? launch_zvc_relu_compress(d_src, n, s, nan_above, d_relu_out, d_dst, dst_capacity, d_table, ws, stream,
-                                            on_device)
-                 : launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, stream, on_device);
-        if (e != cudaSuccess) return CDMA_ERR_CUDA;
-    }
-    if (enqueue_result(ws, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
-    return CDMA_OK;
+    const LaunchCtl ctl = make_launch_ctl(h_result);
+    return compress_launch(d_src, n, dtype, relu, d_relu_out, d_dst, dst_capacity, d_table, ws, ctl, stream, h_result);
 }
 
 int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,
@@ -218,10 +269,11 @@ int cdma_zvc_decompress_async(const void* d_src, uint64_t src_bytes, const uint6
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint64_t* ws = static_cast<uint64_t*>(d_workspace);
 
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return CDMA_ERR_CUDA;
-    if (launch_zvc_decompress(d_src, src_bytes, d_table, n, s, d_dst, ws, stream, !in_host_memory(d_src)) != cudaSuccess)
+    if (n == 0) return result_without_kernel(ws, 0, h_result, stream) == cudaSuccess ? CDMA_OK : CDMA_ERR_CUDA;
+    const LaunchCtl ctl = make_launch_ctl(h_result);
+    if (launch_zvc_decompress(d_src, src_bytes, d_table, n, s, d_dst, ws, ctl, stream, !in_host_memory(d_src)) != cudaSuccess)
         return CDMA_ERR_CUDA;
-    if (enqueue_result(ws, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    if (finish_result(ws, ctl, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
     return CDMA_OK;
 }
 
@@ -250,14 +302,13 @@ int cdma_rle_compress_async(const void* d_src, uint64_t n, int dtype, int layout
     if (overlaps(d_src, n * 4, d_dst, dst_capacity)) return CDMA_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint64_t* ws = static_cast<uint64_t*>(d_workspace);
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * kDescStride * num_tiles_of(n), stream) != cudaSuccess)
-        return CDMA_ERR_CUDA;
     if (n == 0) {
         if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return CDMA_ERR_CUDA;
-    } else if (launch_rle_compress(d_src, n, d_dst, dst_capacity, d_table, ws, stream) != cudaSuccess) {
-        return CDMA_ERR_CUDA;
+        return result_without_kernel(ws, 0, h_result, stream) == cudaSuccess ? CDMA_OK : CDMA_ERR_CUDA;
     }
-    if (enqueue_result(ws, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    const LaunchCtl ctl = make_launch_ctl(h_result);
+    if (launch_rle_compress(d_src, n, d_dst, dst_capacity, d_table, ws, ctl, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    if (finish_result(ws, ctl, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
     return CDMA_OK;
 }
 
@@ -288,9 +339,10 @@ int cdma_rle_decompress_async(const void* d_src, uint64_t src_bytes, const uint6
     if (src_bytes < 4 * chunks || src_bytes > 4 * (n + chunks) || src_bytes % 4 != 0) return CDMA_ERR_CORRUPT_STREAM;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint64_t* ws = static_cast<uint64_t*>(d_workspace);
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return CDMA_ERR_CUDA;
-    if (launch_rle_decompress(d_src, src_bytes, d_table, n, d_dst, ws, stream) != cudaSuccess) return CDMA_ERR_CUDA;
-    if (enqueue_result(ws, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    if (n == 0) return result_without_kernel(ws, 0, h_result, stream) == cudaSuccess ? CDMA_OK : CDMA_ERR_CUDA;
+    const LaunchCtl ctl = make_launch_ctl(h_result);
+    if (launch_rle_decompress(d_src, src_bytes, d_table, n, d_dst, ws, ctl, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    if (finish_result(ws, ctl, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
     return CDMA_OK;
 }
 
@@ -305,6 +357,30 @@ int64_t cdma_rle_decompress(const void* d_src, uint64_t src_bytes, const uint64_
         return -static_cast<int64_t>(CDMA_ERR_CUDA);
     if (result[1] != 0) return -static_cast<int64_t>(result[1]);
     return static_cast<int64_t>(n) * 4;
+}
+
+// Test hook, deliberately not declared in cdma.h: cdma_zvc_compress with one tile
+// that never publishes its look-back descriptor and a short bound on the device-side
+// waits, so that the tiles behind it run into the bound.  Every wait is bounded, the
+// kernel returns normally and the call reports -CDMA_ERR_TIMEOUT; nothing traps or
+// spins without limit.  stall_tile >= the number of tiles stalls nothing.
+int64_t cdma_test_compress_stalled(const void* d_src, uint64_t n, int dtype, void* d_dst, uint64_t dst_capacity,
+                                   uint64_t* d_table, void* d_workspace, uint64_t workspace_bytes,
+                                   void* cuda_stream, uint32_t stall_tile, uint64_t wait_limit_ns) {
+    const int st = check_common(n, dtype, CDMA_NCHW, d_src, d_dst, d_table, d_workspace, workspace_bytes);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (n == 0 || wait_limit_ns == 0 || wait_limit_ns > kWaitLimitNs) return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
+    uint64_t result[2] = {0, 0};
+    LaunchCtl ctl = make_launch_ctl(result);
+    ctl.stall_tile = stall_tile;
+    ctl.wait_limit_ns = wait_limit_ns;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int ls = compress_launch(d_src, n, dtype, false, nullptr, d_dst, dst_capacity, d_table,
+                                   static_cast<uint64_t*>(d_workspace), ctl, stream, result);
+    if (ls != CDMA_OK) return -static_cast<int64_t>(ls);
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (result[1] != 0) return -static_cast<int64_t>(result[1]);
+    return static_cast<int64_t>(result[0]);
 }
 
 void cdma_time_next_kernel(void* start_event, void* stop_event) {

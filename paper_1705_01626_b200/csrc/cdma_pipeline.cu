@@ -3,7 +3,8 @@
 // memory, PRE(n) copies them back and expands them.  The codec kernels run on
 // the caller's compute stream, the copies on a side stream owned by the
 // context; two device staging slots let one tensor's copy overlap the next
-// tensor's kernel.  Host code only: contracts are in include/cdma.h.
+// tensor's kernel.  Host code, plus the small copy kernel of the asynchronous
+// offload; contracts are in include/cdma.h.
 #include <map>
 #include <new>
 #include <unordered_map>
@@ -90,7 +91,34 @@ struct TicketRec {
     uint64_t payload_bytes;
     uint64_t pool_off, pool_bytes;      // region of the pinned pool owned by the ticket
     uint64_t payload_off, table_off;    // where payload and table sit inside the pool
+    // asynchronous offloads: the size is not known when the ticket is handed out
+    bool resolved = true;
+    const uint64_t* res = nullptr;      // pinned {bytes, status} written by the compression kernel
+    cudaEvent_t done = nullptr;         // the ticket's bytes have landed in the pool
 };
+
+// Copy of an offloaded tensor from a device staging slot into the mapped pinned
+// pool, for the case where the host does not know the payload size yet: the
+// kernel reads the size (and the status) the compression kernel left in the
+// slot's workspace and moves exactly that many payload bytes plus the offset
+// table.  A few CTAs saturate the host link; the rest of the GPU stays free for
+// the caller's compute stream.
+constexpr uint32_t kCopyCtas = 48;
+constexpr uint32_t kCopyThreads = 256;
+__global__ void __launch_bounds__(kCopyThreads)
+offload_copy_kernel(const uint64_t* __restrict__ ws, const uint4* __restrict__ payload, uint4* __restrict__ pool_payload,
+                    const uint4* __restrict__ table, uint4* __restrict__ pool_table, uint64_t table_vecs,
+                    uint64_t capacity) {
+    const uint64_t bytes = ws[cdma::kWsBytes];
+    const uint64_t status = ws[cdma::kWsStatus];
+    if (status != 0 || bytes > capacity) return;          // nothing valid to move; the host sees the status
+    const uint64_t vecs = (bytes + 15) / 16;               // the slot and the pool region are padded to 16 bytes
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    for (uint64_t i = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < vecs; i += stride)
+        pool_payload[i] = __ldcs(payload + i);
+    for (uint64_t i = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < table_vecs; i += stride)
+        pool_table[i] = __ldcs(table + i);
+}
 
 }  // namespace
 
@@ -111,6 +139,10 @@ struct cdma_ctx {
     int deferred = 0;
     void* d_dense = nullptr;          // dense staging of the host-buffer calls
     uint64_t dense_bytes = 0;
+    std::vector<uint64_t> unresolved; // asynchronous offload tickets whose size has not been read yet, oldest first
+    std::vector<cudaEvent_t> spare_events;
+    cudaEvent_t pool_read = nullptr;  // last side-stream copy that reads the pinned pool
+    bool pool_read_used = false;
 };
 
 namespace {
@@ -165,6 +197,9 @@ int wait_all(cdma_ctx* ctx) {
     return CDMA_OK;
 }
 
+bool settle_ticket(cdma_ctx* ctx, uint64_t id, bool block);
+void settle_all(cdma_ctx* ctx, bool block);
+
 int ensure_dense(cdma_ctx* ctx, uint64_t bytes) {
     if (bytes <= ctx->dense_bytes) return CDMA_OK;
     if (wait_all(ctx) != CDMA_OK) return CDMA_ERR_CUDA;
@@ -177,6 +212,73 @@ int ensure_dense(cdma_ctx* ctx, uint64_t bytes) {
     }
     ctx->dense_bytes = round_up(bytes, kAlign);
     return CDMA_OK;
+}
+
+cudaEvent_t take_event(cdma_ctx* ctx) {
+    if (!ctx->spare_events.empty()) {
+        cudaEvent_t e = ctx->spare_events.back();
+        ctx->spare_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return e;
+}
+
+// An asynchronous offload hands out its ticket before the payload size exists.  The
+// first caller that needs the size settles the ticket: waits (or, with block = false,
+// only looks) for the ticket's bytes to have landed, reads the size the kernel stored
+// in pinned memory, and gives the unused tail of the worst-case reservation back to
+// the pool.  A ticket whose compression failed is dropped and its status deferred.
+// Returns false if the ticket is still in flight (block = false only).
+bool settle_ticket(cdma_ctx* ctx, uint64_t id, bool block) {
+    auto it = ctx->tickets.find(id);
+    if (it == ctx->tickets.end() || it->second.resolved) return true;
+    TicketRec& rec = it->second;
+    if (block) {
+        if (cudaEventSynchronize(rec.done) != cudaSuccess) cudaGetLastError();
+    } else if (cudaEventQuery(rec.done) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    ctx->spare_events.push_back(rec.done);
+    rec.done = nullptr;
+    rec.resolved = true;
+    for (size_t i = 0; i < ctx->unresolved.size(); ++i)
+        if (ctx->unresolved[i] == id) { ctx->unresolved.erase(ctx->unresolved.begin() + i); break; }
+    const uint64_t status = rec.res[1];
+    if (status != 0) {
+        if (ctx->deferred == 0) ctx->deferred = static_cast<int>(status);
+        ctx->pool.release(rec.pool_off, rec.pool_bytes);
+        ctx->tickets.erase(it);
+        return true;
+    }
+    rec.payload_bytes = rec.res[0];
+    const uint64_t used = (rec.payload_off - rec.pool_off) + rec.payload_bytes;
+    ctx->pool.shrink(rec.pool_off, rec.pool_bytes, used);
+    rec.pool_bytes = used;
+    return true;
+}
+
+void settle_all(cdma_ctx* ctx, bool block) {
+    const std::vector<uint64_t> ids = ctx->unresolved;
+    for (uint64_t id : ids) settle_ticket(ctx, id, block);
+}
+
+// Pool allocation that first gives back what finished asynchronous offloads over-reserved, and
+// waits for the ones still in flight (oldest first) before it reports the pool exhausted.
+bool pool_alloc(cdma_ctx* ctx, uint64_t bytes, uint64_t* off) {
+    if (ctx->pool.alloc(bytes, off)) return true;
+    settle_all(ctx, false);
+    if (ctx->pool.alloc(bytes, off)) return true;
+    while (!ctx->unresolved.empty()) {
+        settle_ticket(ctx, ctx->unresolved.front(), true);
+        if (ctx->pool.alloc(bytes, off)) return true;
+    }
+    return false;
 }
 
 }  // namespace
@@ -210,6 +312,9 @@ int cdma_ctx_create(uint64_t pinned_bytes, uint64_t device_staging_bytes, cdma_c
             cudaMalloc(reinterpret_cast<void**>(&ctx->d_staging), slot_bytes * kSlots) != cudaSuccess) {
             st = CDMA_ERR_OUT_OF_MEMORY; break;
         }
+        if (cudaEventCreateWithFlags(&ctx->pool_read, cudaEventDisableTiming) != cudaSuccess) {
+            st = CDMA_ERR_CUDA; break;
+        }
         for (uint32_t i = 0; i < kSlots && st == CDMA_OK; ++i) {
             ctx->slots[i].base = ctx->d_staging ? ctx->d_staging + i * slot_bytes : nullptr;
             ctx->slots[i].bytes = slot_bytes;
@@ -235,6 +340,10 @@ int cdma_ctx_destroy(cdma_ctx* ctx) {
         if (s.idle) cudaEventDestroy(s.idle);
         if (s.staged) cudaEventDestroy(s.staged);
     }
+    for (auto& kv : ctx->tickets)
+        if (kv.second.done) cudaEventDestroy(kv.second.done);
+    for (cudaEvent_t e : ctx->spare_events) cudaEventDestroy(e);
+    if (ctx->pool_read) cudaEventDestroy(ctx->pool_read);
     if (ctx->d_dense) cudaFree(ctx->d_dense);
     if (ctx->d_staging) cudaFree(ctx->d_staging);
     if (ctx->h_results) cudaFreeHost(ctx->h_results);
@@ -271,7 +380,7 @@ int64_t cdma_offload(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, in
     // exactly C payload bytes and the table cross the link (Section V-D: the
     // compressed size is known on completion and sizes the host allocation)
     TicketRec rec{n, dtype, layout, c, 0, round_up(c, 16) + p.table_bytes, 0, 0};
-    if (!ctx->pool.alloc(rec.pool_bytes, &rec.pool_off) ||
+    if (!pool_alloc(ctx, rec.pool_bytes, &rec.pool_off) ||
         rec.pool_off + rec.pool_bytes > ctx->pool_bytes)
         return -static_cast<int64_t>(CDMA_ERR_OUT_OF_MEMORY);
     rec.payload_off = rec.pool_off;
@@ -291,15 +400,85 @@ int64_t cdma_offload(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, in
     return static_cast<int64_t>(c);
 }
 
+// OFF without a host-side wait (Fig. 2b: the offload of a layer's map overlaps the layers that
+// follow; Section V-D: the size is reported on completion, not needed to start the copy).
+int cdma_offload_async(cdma_ctx* ctx, const void* d_src, uint64_t n, int dtype, int layout, void* compute_stream,
+                       cdma_ticket* out) {
+    if (ctx == nullptr || out == nullptr) return CDMA_ERR_INVALID_ARG;
+    if (cdma_dtype_size(dtype) == 0) return CDMA_ERR_UNSUPPORTED_DTYPE;
+    cudaStream_t compute = static_cast<cudaStream_t>(compute_stream);
+    // keep the ring of pinned result words ahead of the tickets that still point into it
+    while (ctx->pending.size() + ctx->unresolved.size() + 2 >= kResultRing) {
+        if (!ctx->unresolved.empty()) settle_ticket(ctx, ctx->unresolved.front(), true);
+        else if (wait_all(ctx) != CDMA_OK) return CDMA_ERR_CUDA;
+    }
+    Slot& slot = ctx->slots[ctx->next_slot % kSlots];
+    SlotPlan p;
+    if (!plan_slot(slot, n, dtype, &p)) return CDMA_ERR_BUFFER_TOO_SMALL;
+    // the size is not known yet: reserve the most this slot's payload can be; the rest comes back
+    // when the ticket is settled
+    const uint64_t table_room = round_up(p.table_bytes, kAlign);
+    TicketRec rec{n, dtype, layout, 0, 0, table_room + round_up(p.capacity, 16), 0, 0};
+    if (!pool_alloc(ctx, rec.pool_bytes, &rec.pool_off) || rec.pool_off + rec.pool_bytes > ctx->pool_bytes)
+        return CDMA_ERR_OUT_OF_MEMORY;
+    rec.table_off = rec.pool_off;
+    rec.payload_off = rec.pool_off + table_room;
+    void* m_payload = nullptr;
+    void* m_table = nullptr;
+    cudaEvent_t done = take_event(ctx);
+    bool ok = done != nullptr;
+    ok = ok && cudaHostGetDevicePointer(&m_payload, ctx->h_pool + rec.payload_off, 0) == cudaSuccess;
+    ok = ok && cudaHostGetDevicePointer(&m_table, ctx->h_pool + rec.table_off, 0) == cudaSuccess;
+    // the slot's previous copy must have drained before the kernel overwrites it
+    ok = ok && (!slot.used || cudaStreamWaitEvent(compute, slot.idle, 0) == cudaSuccess);
+    uint64_t* res = next_result_words(ctx);
+    int st = ok ? cdma_zvc_compress_async(d_src, n, dtype, layout, p.payload, p.capacity, p.table, p.ws, p.ws_bytes,
+                                          compute, res)
+                : CDMA_ERR_CUDA;
+    if (st == CDMA_OK) {
+        ++ctx->next_slot;
+        slot.used = true;
+        ok = cudaEventRecord(slot.staged, compute) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(ctx->side, slot.staged, 0) == cudaSuccess;
+        if (ok) {
+            offload_copy_kernel<<<kCopyCtas, kCopyThreads, 0, ctx->side>>>(
+                p.ws, reinterpret_cast<const uint4*>(p.payload), static_cast<uint4*>(m_payload),
+                reinterpret_cast<const uint4*>(p.table), static_cast<uint4*>(m_table), (p.table_bytes + 15) / 16,
+                p.capacity);
+            cdma::count_kernel_launch();
+            ok = cudaGetLastError() == cudaSuccess;
+        }
+        // whatever happened, the slot is busy until the work enqueued so far is through
+        cudaEventRecord(slot.idle, ok ? ctx->side : compute);
+        ok = ok && cudaEventRecord(done, ctx->side) == cudaSuccess;
+        if (!ok) st = CDMA_ERR_CUDA;
+    }
+    if (st != CDMA_OK) {
+        cudaGetLastError();
+        if (done) ctx->spare_events.push_back(done);
+        ctx->pool.release(rec.pool_off, rec.pool_bytes);
+        return st;
+    }
+    rec.resolved = false;
+    rec.res = res;
+    rec.done = done;
+    out->id = ctx->next_ticket++;
+    ctx->tickets[out->id] = rec;
+    ctx->unresolved.push_back(out->id);
+    return CDMA_OK;
+}
+
 static int prefetch_enqueue(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream,
                             Slot** used_slot, uint64_t** result, uint64_t* dense_bytes) {
     if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
+    settle_ticket(ctx, ticket.id, true);      // an asynchronous offload's size is needed now
     auto it = ctx->tickets.find(ticket.id);
     if (it == ctx->tickets.end()) return CDMA_ERR_BAD_TICKET;
     const TicketRec rec = it->second;
     cudaStream_t compute = static_cast<cudaStream_t>(compute_stream);
-    if (ctx->pending.size() + 2 >= kResultRing) {
+    if (ctx->pending.size() + ctx->unresolved.size() + 2 >= kResultRing) {
         if (wait_all(ctx) != CDMA_OK) return CDMA_ERR_CUDA;
+        settle_all(ctx, true);
     }
     Slot& slot = ctx->slots[ctx->next_slot++ % kSlots];
     SlotPlan p;
@@ -314,7 +493,11 @@ static int prefetch_enqueue(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void
                           ctx->side) == cudaSuccess;
     ok &= cudaEventRecord(slot.staged, ctx->side) == cudaSuccess;
     ok &= cudaStreamWaitEvent(compute, slot.staged, 0) == cudaSuccess;
+    // the pool region is given back below while this copy may still be reading it: whoever
+    // writes the pool from another stream waits for this event first
+    ok &= cudaEventRecord(ctx->pool_read, ctx->side) == cudaSuccess;
     if (!ok) return CDMA_ERR_CUDA;
+    ctx->pool_read_used = true;
     slot.used = true;
     cudaEventRecord(slot.idle, ctx->side);
     uint64_t* res = next_result_words(ctx);
@@ -322,8 +505,9 @@ static int prefetch_enqueue(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void
                                              rec.layout, d_dst, p.ws, p.ws_bytes, compute, res);
     if (st != CDMA_OK) return st;   // the ticket stays valid: nothing was consumed
     if (cudaEventRecord(slot.idle, compute) != cudaSuccess) return CDMA_ERR_CUDA;
-    // Later copies into this pinned region are enqueued on the same side
-    // stream, behind the copy just issued, so the region can be recycled now.
+    // The region can be recycled now: later copies into it are enqueued on the same
+    // side stream, behind the copy just issued, and a kernel that writes the pool from
+    // the caller's stream waits for pool_read first.
     ctx->pool.release(rec.pool_off, rec.pool_bytes);
     ctx->tickets.erase(it);
     *used_slot = &slot;
@@ -370,7 +554,7 @@ int64_t cdma_offload_direct(cdma_ctx* ctx, const void* d_src, uint64_t n, int dt
     const uint64_t table_bytes = 8 * cdma_zvc_table_entries(n);
     const uint64_t cap = cdma_zvc_max_compressed_bytes(n, dtype);
     TicketRec rec{n, dtype, layout, 0, 0, round_up(table_bytes, kAlign) + cap, 0, 0};
-    if (!ctx->pool.alloc(rec.pool_bytes, &rec.pool_off) || rec.pool_off + rec.pool_bytes > ctx->pool_bytes)
+    if (!pool_alloc(ctx, rec.pool_bytes, &rec.pool_off) || rec.pool_off + rec.pool_bytes > ctx->pool_bytes)
         return -static_cast<int64_t>(CDMA_ERR_OUT_OF_MEMORY);
     rec.table_off = rec.pool_off;
     rec.payload_off = rec.pool_off + round_up(table_bytes, kAlign);
@@ -382,7 +566,10 @@ int64_t cdma_offload_direct(cdma_ctx* ctx, const void* d_src, uint64_t n, int dt
         ctx->pool.release(rec.pool_off, rec.pool_bytes);
         return -static_cast<int64_t>(CDMA_ERR_CUDA);
     }
-    if (slot.used && cudaStreamWaitEvent(compute, slot.idle, 0) != cudaSuccess) {
+    // the kernel writes the pool from the caller's stream: a region recycled by an earlier
+    // prefetch may still be read by that prefetch's copy on the side stream
+    if ((slot.used && cudaStreamWaitEvent(compute, slot.idle, 0) != cudaSuccess) ||
+        (ctx->pool_read_used && cudaStreamWaitEvent(compute, ctx->pool_read, 0) != cudaSuccess)) {
         ctx->pool.release(rec.pool_off, rec.pool_bytes);
         return -static_cast<int64_t>(CDMA_ERR_CUDA);
     }
@@ -413,6 +600,7 @@ int64_t cdma_offload_direct(cdma_ctx* ctx, const void* d_src, uint64_t n, int dt
 
 int64_t cdma_prefetch_direct(cdma_ctx* ctx, cdma_ticket ticket, void* d_dst, void* compute_stream) {
     if (ctx == nullptr) return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
+    settle_ticket(ctx, ticket.id, true);
     auto it = ctx->tickets.find(ticket.id);
     if (it == ctx->tickets.end()) return -static_cast<int64_t>(CDMA_ERR_BAD_TICKET);
     const TicketRec rec = it->second;
@@ -447,6 +635,7 @@ int cdma_ctx_synchronize(cdma_ctx* ctx) {
     if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
     const int st = wait_all(ctx);
     if (st != CDMA_OK) return st;
+    settle_all(ctx, true);
     const int d = ctx->deferred;
     ctx->deferred = 0;
     return d;
@@ -454,6 +643,7 @@ int cdma_ctx_synchronize(cdma_ctx* ctx) {
 
 int cdma_ticket_info(cdma_ctx* ctx, cdma_ticket ticket, uint64_t* payload_bytes, uint64_t* n) {
     if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
+    settle_ticket(ctx, ticket.id, true);
     auto it = ctx->tickets.find(ticket.id);
     if (it == ctx->tickets.end()) return CDMA_ERR_BAD_TICKET;
     if (payload_bytes) *payload_bytes = it->second.payload_bytes;
@@ -463,6 +653,7 @@ int cdma_ticket_info(cdma_ctx* ctx, cdma_ticket ticket, uint64_t* payload_bytes,
 
 int cdma_ticket_host_view(cdma_ctx* ctx, cdma_ticket ticket, const void** h_payload, const uint64_t** h_table) {
     if (ctx == nullptr) return CDMA_ERR_INVALID_ARG;
+    settle_ticket(ctx, ticket.id, true);
     auto it = ctx->tickets.find(ticket.id);
     if (it == ctx->tickets.end()) return CDMA_ERR_BAD_TICKET;
     // copies into the pool are asynchronous on the side stream: let them land before the host looks

@@ -14,10 +14,8 @@
 //
 // Host code must not hand the array's name to a kernel: in host code the name
 // is only a host-side stand-in for the symbol, not a device address.  The
-// device address is looked up once per device with cudaGetSymbolAddress, with
-// that device current, and that pointer is what the kernel receives.
-#include <mutex>
-
+// device address is looked up with cudaGetSymbolAddress, with the calling
+// device current, and that pointer is what the kernel receives.
 #include "zvc_common.cuh"
 
 namespace {
@@ -30,25 +28,20 @@ constexpr uint64_t kStaticWsBytes =
 
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 
-constexpr int kMaxDevices = 64;
-std::mutex g_setup_mutex;
-uint64_t* g_ws_ptr[kMaxDevices] = {};
-
-// Device address of the workspace on the current device; looked up on the
-// first call made with that device current.  Returns nullptr on failure.
-uint64_t* static_ws_for_current_device() {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-    std::lock_guard<std::mutex> lock(g_setup_mutex);
-    if (g_ws_ptr[dev] == nullptr) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || p == nullptr) {
-            cudaGetLastError();
-            return nullptr;
-        }
-        g_ws_ptr[dev] = static_cast<uint64_t*>(p);
+// Device address of the workspace on the current device.  Looked up on every call
+// (after the first time on a device this is a table look-up inside the runtime),
+// so that a pointer from before a cudaDeviceReset is never reused.  The first
+// look-up on a device loads this module, which is when the array's memory is
+// reserved there: it can fail for lack of memory on a full device.
+int static_ws_for_current_device(uint64_t** out) {
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_static_ws);
+    if (e != cudaSuccess || p == nullptr) {
+        (void)cudaGetLastError();
+        return e == cudaErrorMemoryAllocation ? CDMA_ERR_OUT_OF_MEMORY : CDMA_ERR_CUDA;
     }
-    return g_ws_ptr[dev];
+    *out = static_cast<uint64_t*>(p);
+    return CDMA_OK;
 }
 
 inline bool aligned_to(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -74,20 +67,25 @@ extern "C" int64_t cdma_zvc_compress_static_ws(const void* d_src, uint64_t n, in
         if (n != 0 && dst_capacity != 0 && a0 < b0 + dst_capacity && b0 < a0 + n * s)
             return -static_cast<int64_t>(CDMA_ERR_INVALID_ARG);
     }
-    uint64_t* ws = static_ws_for_current_device();
-    if (ws == nullptr) return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    uint64_t* ws = nullptr;
+    const int ws_status = static_ws_for_current_device(&ws);
+    if (ws_status != CDMA_OK) return -static_cast<int64_t>(ws_status);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
-    // The array keeps whatever the previous call left: ticket, result words and
-    // the descriptors of every tile this call uses must start at zero.
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes + 8 * kDescStride * num_tiles_of(n), stream) != cudaSuccess)
-        return -static_cast<int64_t>(CDMA_ERR_CUDA);
-    if (n == 0) {
-        if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess) return -static_cast<int64_t>(CDMA_ERR_CUDA);
-    } else if (launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, stream) != cudaSuccess) {
-        return -static_cast<int64_t>(CDMA_ERR_CUDA);
-    }
+    // The array keeps whatever the previous call left.  Nothing in it has to start
+    // at zero: the look-back descriptors of this launch carry a tag of their own,
+    // and the result words are written by the launch before they are read.
     uint64_t result[2] = {0, 0};
+    LaunchCtl ctl = make_launch_ctl(nullptr);            // result words come back by the copy below
+    if (n == 0) {
+        if (cudaMemsetAsync(d_table, 0, 8, stream) != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess)
+            return -static_cast<int64_t>(CDMA_ERR_CUDA);
+        return 0;
+    }
+    // a source in page-locked host memory is read over the host link: no L2 prefetches for it
+    if (launch_zvc_compress(d_src, n, s, d_dst, dst_capacity, d_table, ws, ctl, stream, !in_host_memory(d_src)) !=
+        cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
     if (cudaMemcpyAsync(result, ws + kWsBytes, 16, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess)
         return -static_cast<int64_t>(CDMA_ERR_CUDA);

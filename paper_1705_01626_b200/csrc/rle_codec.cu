@@ -28,8 +28,8 @@ constexpr uint32_t kBig = 0x7fffffffu;
 
 __global__ void __launch_bounds__(kTileThreads, 4)
 rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
-                    uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
-                    uint64_t num_chunks) {
+                    uint64_t* __restrict__ table, uint64_t* __restrict__ ws, const LaunchCtl ctl,
+                    uint32_t num_tiles, uint64_t num_chunks) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     uint32_t* s_tile = reinterpret_cast<uint32_t*>(smem_raw);       // the tile's records, contiguous
     __shared__ uint32_t s_chunk_units[kTileChunks];
@@ -41,7 +41,6 @@ rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __res
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t lt = lanemask_lt();
-    uint64_t* desc = ws + kWsDescriptors;
     const uint32_t tile = blockIdx.x;          // block-index order, as in the zero-value kernel
     if (tile >= num_tiles) return;
 
@@ -92,9 +91,7 @@ rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __res
     uint64_t tile_bytes = 0;
     if (warp == 0) {
         tile_bytes = static_cast<uint64_t>(__reduce_add_sync(0xffffffffu, cu)) * 4u;
-        if (lane == 0)
-            st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride,
-                           (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+        if (lane == 0) publish_aggregate(ws, ctl, tile, tile_bytes);
     }
 
     // ---- 2. assemble the chunk's records in the staged tile --------------------------
@@ -128,35 +125,15 @@ rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __res
     if (trailing && lane == 0) st[units - 1] = nelem - 1u - static_cast<uint32_t>(last_nz);   // zeros only
 
     // ---- 3. the tile's place in the stream ------------------------------------------
-    if (warp == 0) {
-        LookbackResult lb{0, false};
-        if (tile != 0) {
-            lb = lookback_walk(desc, ws, tile);
-            if (lane == 0)
-                st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride,
-                               lb.failed ? kDescError : (kDescPrefix | (lb.exclusive + tile_bytes)));
-        }
-        if (lane == 0) {
-            s_base = lb.exclusive;
-            s_failed = lb.failed ? 1u : 0u;
-            const uint64_t end_bytes = lb.exclusive + tile_bytes;
-            s_room = static_cast<uint32_t>((cap >= end_bytes ? tile_bytes : (cap > lb.exclusive ? cap - lb.exclusive : 0)) / 4u);
-            if (!lb.failed) {
-                if (tile == num_tiles - 1) {
-                    table[num_chunks] = end_bytes;
-                    ws[kWsBytes] = end_bytes;
-                }
-                if (end_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
-            }
-        }
-    }
+    if (warp == 0)
+        resolve_tile(ws, ctl, tile, num_tiles, tile_bytes, cap, table, num_chunks, &s_base, &s_failed, &s_room);
     __syncthreads();
     if (s_failed) return;
 
     // ---- 4. the CTA writes the tile's words to their place, below cap ----------------
     const uint64_t first_unit = s_base / 4u;
     if (lane == 0 && chunk < num_chunks) table[chunk] = (first_unit + chunk_off) * 4u;
-    const uint32_t room = s_room;
+    const uint32_t room = s_room / 4u;           // whole words below the capacity
     uint32_t* out = reinterpret_cast<uint32_t*>(dst) + first_unit;
     for (uint32_t u = threadIdx.x; u < room; u += kTileThreads) out[u] = s_tile[u];
 }
@@ -165,7 +142,8 @@ constexpr uint32_t kRleDecWarps = 8;
 
 __global__ void __launch_bounds__(32 * kRleDecWarps)
 rle_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const uint64_t* __restrict__ table,
-                      uint64_t n, uint32_t* __restrict__ dst, uint64_t* __restrict__ ws, uint64_t num_chunks) {
+                      uint64_t n, uint32_t* __restrict__ dst, uint64_t* __restrict__ ws, const LaunchCtl ctl,
+                      uint64_t num_chunks) {
     // staged payload (16-byte phase in front)
     constexpr uint32_t kStageWords = kRleMaxChunkUnits + 4 + 3;
     __shared__ __align__(16) uint32_t s_stage[kRleDecWarps][(kStageWords + 3) / 4 * 4];
@@ -173,7 +151,7 @@ rle_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
     const uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * kRleDecWarps + warp;
-    if (blockIdx.x == 0 && threadIdx.x == 0) ws[kWsBytes] = n * 4u;
+    if (blockIdx.x == 0 && threadIdx.x == 0) init_decode_result(ws, ctl, n * 4u);
     if (chunk >= num_chunks) return;
     const uint64_t e0 = chunk * kChunk;
     const uint32_t nelem = (n - e0 < kChunk) ? static_cast<uint32_t>(n - e0) : kChunk;
@@ -187,7 +165,7 @@ rle_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const
     if (chunk == 0 && lo != 0) ok = false;
     if (chunk == num_chunks - 1 && hi != src_bytes) ok = false;
     if (!ok) {
-        if (lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+        if (lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
         return;
     }
 
@@ -246,22 +224,22 @@ rle_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const
     }
     bad |= zero_literal != 0u;
     bad = __any_sync(0xffffffffu, bad) || p != end;
-    if (bad && lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+    if (bad && lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
 }
 
 }  // namespace
 
 cudaError_t launch_rle_compress(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
-                                uint64_t* d_ws, cudaStream_t stream) {
+                                uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream) {
     const uint64_t chunks = num_chunks_of(n);
     const uint64_t tiles = num_tiles_of(n);
     if (tiles == 0) return cudaSuccess;
     constexpr uint32_t kSmem = kTileChunks * kRleMaxChunkUnits * 4;
-    const cudaError_t e = cudaFuncSetAttribute(rle_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    const cudaError_t e = opt_in_shared_memory(reinterpret_cast<const void*>(rle_compress_kernel), kSmem);
     if (e != cudaSuccess) return e;
     timing_before_launch(stream);
     rle_compress_kernel<<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
-        static_cast<const uint32_t*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
+        static_cast<const uint32_t*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws, ctl,
         static_cast<uint32_t>(tiles), chunks);
     timing_after_launch(stream);
     count_kernel_launch();
@@ -269,14 +247,14 @@ cudaError_t launch_rle_compress(const void* d_src, uint64_t n, void* d_dst, uint
 }
 
 cudaError_t launch_rle_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
-                                  void* d_dst, uint64_t* d_ws, cudaStream_t stream) {
+                                  void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream) {
     const uint64_t chunks = num_chunks_of(n);
     if (chunks == 0) return cudaSuccess;
     const dim3 grid(static_cast<unsigned>((chunks + kRleDecWarps - 1) / kRleDecWarps));
     timing_before_launch(stream);
     rle_decompress_kernel<<<grid, 32 * kRleDecWarps, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes,
                                                                    d_table, n, static_cast<uint32_t*>(d_dst), d_ws,
-                                                                   chunks);
+                                                                   ctl, chunks);
     timing_after_launch(stream);
     count_kernel_launch();
     return cudaGetLastError();

@@ -41,14 +41,9 @@ __device__ __forceinline__ void load4(const uint16_t* p, uint32_t (&e)[4]) {
 // about half a CTA lifetime from now (5 CTAs x 148 SMs are resident at a time).
 // Asking L2 for it now turns that CTA's DRAM-latency load phase into L2 hits;
 // every line is still fetched from DRAM exactly once.
-#ifndef CDMA_PREFETCH_AHEAD
-#define CDMA_PREFETCH_AHEAD 370
-#endif
-constexpr uint32_t kPrefetchAhead = CDMA_PREFETCH_AHEAD;
-constexpr uint32_t kTileBytes = kTileChunks * kChunk * 4;      // 32 KB for either element width
+constexpr uint32_t kPrefetchAhead = 370;
 
 __device__ __forceinline__ void prefetch_future_tile(const void* src, uint64_t total_bytes, uint32_t tile) {
-    if (kPrefetchAhead == 0) return;
     const uint64_t off = (static_cast<uint64_t>(tile) + kPrefetchAhead) * kTileBytes + 128ull * threadIdx.x;
     if (off + 128 <= total_bytes)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const uint8_t*>(src) + off));
@@ -133,7 +128,7 @@ template <bool RELU, bool FULL>
 __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ src, uint64_t n,
                                                   uint8_t* __restrict__ dst, uint64_t cap,
                                                   uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
-                                                  uint32_t num_tiles, uint64_t num_chunks,
+                                                  const LaunchCtl& ctl, uint32_t num_tiles, uint64_t num_chunks,
                                                   uint32_t* __restrict__ relu_out, uint32_t tile) {
     constexpr uint32_t S = 4;
     extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -146,7 +141,6 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t lt = lanemask_lt();
-    uint64_t* desc = ws + kWsDescriptors;
 
     // ---- load the warp's chunk: 32 loads per lane, all in flight --------------
     const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunks + warp;
@@ -192,8 +186,7 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
     if (warp == 0) {
         tile_bytes = static_cast<uint64_t>(__reduce_add_sync(0xffffffffu, cu)) * S;
         // the tile's size is public before any record is assembled
-        if (lane == 0)
-            st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride, (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+        if (lane == 0) publish_aggregate(ws, ctl, tile, tile_bytes);
     }
 
     // ---- 2. assemble the chunk's records at its place in the staged tile ------
@@ -202,36 +195,15 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
     assemble_windows<0>(a, e, FULL ? kChunkWindows : nwin, lt);
 
     // ---- 3. the tile's place in the stream ------------------------------------
-    if (warp == 0) {
-        LookbackResult lb{0, false};
-        if (tile != 0) {
-            lb = lookback_walk(desc, ws, tile);
-            if (lane == 0)
-                st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride, lb.failed ? kDescError
-                                                      : (kDescPrefix | (lb.exclusive + tile_bytes)));
-        }
-        if (lane == 0) {
-            s_base = lb.exclusive;
-            s_failed = lb.failed ? 1u : 0u;
-            // units of this tile that fit below the capacity
-            const uint64_t end_bytes = lb.exclusive + tile_bytes;
-            s_room = static_cast<uint32_t>((cap >= end_bytes ? tile_bytes : (cap > lb.exclusive ? cap - lb.exclusive : 0)) / S);
-            if (!lb.failed) {
-                if (tile == num_tiles - 1) {
-                    table[num_chunks] = end_bytes;
-                    ws[kWsBytes] = end_bytes;
-                }
-                if (end_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
-            }
-        }
-    }
+    if (warp == 0)
+        resolve_tile(ws, ctl, tile, num_tiles, tile_bytes, cap, table, num_chunks, &s_base, &s_failed, &s_room);
     __syncthreads();
     if (s_failed) return;
 
     // ---- 4. the CTA writes the tile's bytes to their place, below cap ---------
     const uint64_t first_unit = s_base / S;
     if (lane == 0 && chunk < num_chunks) table[chunk] = (first_unit + chunk_off) * S;
-    const uint32_t room = s_room;
+    const uint32_t room = s_room / S;                            // whole units below the capacity
     // Row r of the copy is the aligned 128-byte line r of the destination that the
     // tile touches: thread t moves unit u = t - mis + r * kTileThreads, where mis is
     // how far the tile's first unit sits inside its line; only row 0 can have u < 0.
@@ -256,8 +228,8 @@ __device__ __forceinline__ void compress_tile_u32(const uint32_t* __restrict__ s
 template <typename T, bool RELU>
 __global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
 zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst, uint64_t cap,
-                    uint64_t* __restrict__ table, uint64_t* __restrict__ ws, uint32_t num_tiles,
-                    uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above,
+                    uint64_t* __restrict__ table, uint64_t* __restrict__ ws, const LaunchCtl ctl,
+                    uint32_t num_tiles, uint64_t num_chunks, T* __restrict__ relu_out, uint32_t nan_above,
                     uint64_t prefetch_bytes) {
     static_assert(sizeof(T) == 4, "2-byte elements have a kernel of their own");
     // Tile = block index.  Thread blocks are dispatched in increasing index order,
@@ -268,9 +240,9 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     if (tile >= num_tiles) return;
     prefetch_future_tile(src, prefetch_bytes, tile);
     if ((static_cast<uint64_t>(tile) + 1) * (kTileChunks * kChunk) <= n)
-        compress_tile_u32<RELU, true>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, tile);
+        compress_tile_u32<RELU, true>(src, n, dst, cap, table, ws, ctl, num_tiles, num_chunks, relu_out, tile);
     else
-        compress_tile_u32<RELU, false>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, tile);
+        compress_tile_u32<RELU, false>(src, n, dst, cap, table, ws, ctl, num_tiles, num_chunks, relu_out, tile);
 }
 
 // 2-byte elements: a lane holds 8 consecutive elements (one 16-byte load), so a
@@ -355,7 +327,7 @@ template <bool RELU, bool FULL>
 __device__ __forceinline__ void compress_tile_u16(const uint16_t* __restrict__ src, uint64_t n,
                                                   uint8_t* __restrict__ dst, uint64_t cap,
                                                   uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
-                                                  uint32_t num_tiles, uint64_t num_chunks,
+                                                  const LaunchCtl& ctl, uint32_t num_tiles, uint64_t num_chunks,
                                                   uint16_t* __restrict__ relu_out, uint32_t nan_above,
                                                   uint32_t tile) {
     constexpr uint32_t S = 2;
@@ -367,7 +339,6 @@ __device__ __forceinline__ void compress_tile_u16(const uint16_t* __restrict__ s
 
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
-    uint64_t* desc = ws + kWsDescriptors;
 
     // ---- load the warp's two chunks ------------------------------------------
     uint32_t nwin[2] = {kChunkWindows, kChunkWindows};
@@ -437,9 +408,7 @@ __device__ __forceinline__ void compress_tile_u16(const uint16_t* __restrict__ s
     if (warp == 0) {
         tile_bytes = static_cast<uint64_t>(__reduce_add_sync(0xffffffffu, cu)) * S;
         // the tile's size is public before any record is assembled
-        if (lane == 0)
-            st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride,
-                           (tile == 0 ? kDescPrefix : kDescAggregate) | tile_bytes);
+        if (lane == 0) publish_aggregate(ws, ctl, tile, tile_bytes);
     }
 
     // ---- 2. assemble both chunks' records at their place in the staged tile ----
@@ -448,29 +417,8 @@ __device__ __forceinline__ void compress_tile_u16(const uint16_t* __restrict__ s
     assemble_chunk_u16<FULL>(s_addr + S * (chunk_off + units[0]), bits[1], w[1], lane, nwin[1]);
 
     // ---- 3. the tile's place in the stream ------------------------------------
-    if (warp == 0) {
-        LookbackResult lb{0, false};
-        if (tile != 0) {
-            lb = lookback_walk(desc, ws, tile);
-            if (lane == 0)
-                st_relaxed_u64(desc + static_cast<uint64_t>(tile) * kDescStride,
-                               lb.failed ? kDescError : (kDescPrefix | (lb.exclusive + tile_bytes)));
-        }
-        if (lane == 0) {
-            s_base = lb.exclusive;
-            s_failed = lb.failed ? 1u : 0u;
-            // bytes of this tile that fit below the capacity (whole units)
-            const uint64_t end_bytes = lb.exclusive + tile_bytes;
-            s_room = static_cast<uint32_t>((cap >= end_bytes ? tile_bytes : (cap > lb.exclusive ? cap - lb.exclusive : 0)) / S) * S;
-            if (!lb.failed) {
-                if (tile == num_tiles - 1) {
-                    table[num_chunks] = end_bytes;
-                    ws[kWsBytes] = end_bytes;
-                }
-                if (end_bytes > cap) report_status(ws, CDMA_ERR_BUFFER_TOO_SMALL);
-            }
-        }
-    }
+    if (warp == 0)
+        resolve_tile(ws, ctl, tile, num_tiles, tile_bytes, cap, table, num_chunks, &s_base, &s_failed, &s_room);
     __syncthreads();
     if (s_failed) return;
 
@@ -480,7 +428,7 @@ __device__ __forceinline__ void compress_tile_u16(const uint16_t* __restrict__ s
         const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunksU16 + 2 * warp + lane;
         if (chunk < num_chunks) table[chunk] = base + S * (chunk_off + (lane ? units[0] : 0u));
     }
-    const uint32_t room = s_room;                                   // bytes, whole units
+    const uint32_t room = s_room & ~1u;                             // bytes, whole units
     // The payload is only 2-byte aligned.  A halfword in front brings the destination
     // to a 4-byte boundary; the body goes out as 32-bit words, each warp store one
     // aligned 128-byte line; a halfword may remain at the end.  When the head halfword
@@ -513,36 +461,33 @@ __device__ __forceinline__ void compress_tile_u16(const uint16_t* __restrict__ s
     }
 }
 
-#ifndef CDMA_MIN_CTAS_U16
-#define CDMA_MIN_CTAS_U16 CDMA_MIN_CTAS
-#endif
 template <bool RELU>
-__global__ void __launch_bounds__(kTileThreads, CDMA_MIN_CTAS_U16)
+__global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
 zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* __restrict__ dst,
                         uint64_t cap, uint64_t* __restrict__ table, uint64_t* __restrict__ ws,
-                        uint32_t num_tiles, uint64_t num_chunks, uint16_t* __restrict__ relu_out,
+                        const LaunchCtl ctl, uint32_t num_tiles, uint64_t num_chunks, uint16_t* __restrict__ relu_out,
                         uint32_t nan_above, uint64_t prefetch_bytes) {
     const uint32_t tile = blockIdx.x;     // block-index order, as in the 4-byte kernel
     if (tile >= num_tiles) return;
     prefetch_future_tile(src, prefetch_bytes, tile);
     if ((static_cast<uint64_t>(tile) + 1) * (kTileChunksU16 * kChunk) <= n)
-        compress_tile_u16<RELU, true>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, nan_above, tile);
+        compress_tile_u16<RELU, true>(src, n, dst, cap, table, ws, ctl, num_tiles, num_chunks, relu_out, nan_above, tile);
     else
-        compress_tile_u16<RELU, false>(src, n, dst, cap, table, ws, num_tiles, num_chunks, relu_out, nan_above, tile);
+        compress_tile_u16<RELU, false>(src, n, dst, cap, table, ws, ctl, num_tiles, num_chunks, relu_out, nan_above, tile);
 }
 
 template <typename T, uint32_t TILE_CHUNKS, typename Kernel>
 cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_dst, uint64_t cap,
-                         uint64_t* d_table, uint64_t* d_ws, void* d_relu_out, uint32_t nan_above,
-                         cudaStream_t stream, bool src_on_device) {
+                         uint64_t* d_table, uint64_t* d_ws, const LaunchCtl& ctl, void* d_relu_out,
+                         uint32_t nan_above, cudaStream_t stream, bool src_on_device) {
     constexpr uint32_t kSmem = TILE_CHUNKS * (4 * kChunkWindows + sizeof(T) * kChunk);
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-    if (e != cudaSuccess) return e;
+    const cudaError_t oe = opt_in_shared_memory(reinterpret_cast<const void*>(kernel), kSmem);
+    if (oe != cudaSuccess) return oe;
     const uint64_t chunks = num_chunks_of(n);
     const uint64_t tiles = (chunks + TILE_CHUNKS - 1) / TILE_CHUNKS;   // never more than num_tiles_of(n)
     timing_before_launch(stream);
     kernel<<<static_cast<unsigned>(tiles), kTileThreads, kSmem, stream>>>(
-        static_cast<const T*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws,
+        static_cast<const T*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws, ctl,
         static_cast<uint32_t>(tiles), chunks, static_cast<T*>(d_relu_out), nan_above,
         src_on_device ? n * sizeof(T) : 0ull);
     timing_after_launch(stream);
@@ -552,29 +497,30 @@ cudaError_t launch_typed(Kernel kernel, const void* d_src, uint64_t n, void* d_d
 }  // namespace
 
 cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst,
-                                uint64_t cap, uint64_t* d_table, uint64_t* d_ws,
+                                uint64_t cap, uint64_t* d_table, uint64_t* d_ws, const LaunchCtl& ctl,
                                 cudaStream_t stream, bool src_on_device) {
     if (num_tiles_of(n) == 0) return cudaSuccess;
     const cudaError_t e =
         (elem_size == 4)
             ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t, false>, d_src, n, d_dst, cap,
-                                                  d_table, d_ws, nullptr, 0, stream, src_on_device)
+                                                  d_table, d_ws, ctl, nullptr, 0, stream, src_on_device)
             : launch_typed<uint16_t, kTileChunksU16>(zvc_compress_kernel_u16<false>, d_src, n, d_dst, cap,
-                                                     d_table, d_ws, nullptr, 0, stream, src_on_device);
+                                                     d_table, d_ws, ctl, nullptr, 0, stream, src_on_device);
     count_kernel_launch();
     return e;
 }
 
 cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
                                      void* d_relu_out, void* d_dst, uint64_t cap, uint64_t* d_table,
-                                     uint64_t* d_ws, cudaStream_t stream, bool src_on_device) {
+                                     uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream,
+                                     bool src_on_device) {
     if (num_tiles_of(n) == 0) return cudaSuccess;
     const cudaError_t e =
         (elem_size == 4)
             ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t, true>, d_src, n, d_dst, cap,
-                                                  d_table, d_ws, d_relu_out, nan_above, stream, src_on_device)
+                                                  d_table, d_ws, ctl, d_relu_out, nan_above, stream, src_on_device)
             : launch_typed<uint16_t, kTileChunksU16>(zvc_compress_kernel_u16<true>, d_src, n, d_dst, cap,
-                                                     d_table, d_ws, d_relu_out, nan_above, stream, src_on_device);
+                                                     d_table, d_ws, ctl, d_relu_out, nan_above, stream, src_on_device);
     count_kernel_launch();
     return e;
 }

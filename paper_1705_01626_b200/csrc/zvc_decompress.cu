@@ -21,10 +21,7 @@ namespace {
 
 constexpr uint32_t kDecWarps = 8;
 constexpr uint32_t kDecThreads = 32 * kDecWarps;
-#ifndef CDMA_DEC_PREFETCH_CTAS
-#define CDMA_DEC_PREFETCH_CTAS 888
-#endif
-constexpr uint32_t kPrefetchAheadCtas = CDMA_DEC_PREFETCH_CTAS;   // 6 CTAs x 148 SMs resident at a time
+constexpr uint32_t kPrefetchAheadCtas = 888;   // 6 CTAs x 148 SMs resident at a time
 
 __device__ __forceinline__ void store4(uint32_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     __stcs(reinterpret_cast<uint4*>(p), make_uint4(a, b, c, d));
@@ -108,7 +105,7 @@ template <typename T, bool PREFETCH>
 __global__ void __launch_bounds__(kDecThreads, 6)
 zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
                       const uint64_t* __restrict__ table, uint64_t n, T* __restrict__ dst,
-                      uint64_t* __restrict__ ws, uint64_t num_chunks) {
+                      uint64_t* __restrict__ ws, const LaunchCtl ctl, uint64_t num_chunks) {
     constexpr uint32_t S = sizeof(T);
     constexpr uint32_t MU = 4 / S;                               // units of T per mask
     constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
@@ -125,7 +122,7 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
     const uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * kDecWarps + warp;
-    if (blockIdx.x == 0 && threadIdx.x == 0) ws[kWsBytes] = n * S;
+    if (blockIdx.x == 0 && threadIdx.x == 0) init_decode_result(ws, ctl, n * S);
     if (chunk >= num_chunks) return;
 
     const uint64_t e0 = chunk * kChunk;
@@ -141,7 +138,7 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
     if (chunk == 0 && lo != 0) ok = false;
     if (chunk == num_chunks - 1 && hi != src_bytes) ok = false;
     if (!ok) {
-        if (lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+        if (lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
         return;
     }
 
@@ -171,7 +168,7 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
     // Nothing depends on this and every line still comes from DRAM exactly once.
     // Worth its instructions only where the payload is a sizeable part of the traffic:
     // the launcher picks this variant by the payload-to-dense ratio.
-    if (PREFETCH && kPrefetchAheadCtas != 0) {
+    if (PREFETCH) {
         const uint64_t cf = chunk + static_cast<uint64_t>(kPrefetchAheadCtas) * kDecWarps;
         if (cf < num_chunks) {
             const uint64_t flo = __ldg(table + cf);
@@ -227,7 +224,7 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
         }
     }
     if (!bad && p != end) bad = true;
-    if (bad && lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+    if (bad && lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
 }
 
 // 2-byte elements.  With half the bytes per element the kernel is bound by
@@ -304,22 +301,15 @@ __constant__ uint2 kExpandU16[16] = {
 
 // t[] takes 4.8 KB per warp, so shared memory allows 46-48 warps per SM; CTAs of 2 warps
 // retire and refill most smoothly (4 warps: 2 % slower, 8 warps: 10 %).
-#ifndef CDMA_DEC16_WARPS
-#define CDMA_DEC16_WARPS 2
-#endif
-#ifndef CDMA_DEC16_MINB
-#define CDMA_DEC16_MINB 22
-#endif
-#ifndef CDMA_DEC16_PREFETCH
-#define CDMA_DEC16_PREFETCH 3256          // 22 CTAs x 148 SMs resident at a time
-#endif
-constexpr uint32_t kDec16Warps = CDMA_DEC16_WARPS;
+constexpr uint32_t kDec16Warps = 2;
+constexpr uint32_t kDec16MinCtas = 22;
+constexpr uint32_t kDec16PrefetchCtas = 3256;          // 22 CTAs x 148 SMs resident at a time
 
 template <bool PREFETCH>
-__global__ void __launch_bounds__(32 * kDec16Warps, CDMA_DEC16_MINB)
+__global__ void __launch_bounds__(32 * kDec16Warps, kDec16MinCtas)
 zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
                           const uint64_t* __restrict__ table, uint64_t n, uint16_t* __restrict__ dst,
-                          uint64_t* __restrict__ ws, uint64_t num_chunks) {
+                          uint64_t* __restrict__ ws, const LaunchCtl ctl, uint64_t num_chunks) {
     constexpr uint32_t S = 2, MU = 2;
     __shared__ __align__(32) uint32_t s_t[kDec16Warps][kU16Entries];
     __shared__ uint2 s_expand[16];
@@ -329,7 +319,7 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
     const uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * kDec16Warps + warp;
-    if (blockIdx.x == 0 && threadIdx.x == 0) ws[kWsBytes] = n * S;
+    if (blockIdx.x == 0 && threadIdx.x == 0) init_decode_result(ws, ctl, n * S);
     if (chunk >= num_chunks) return;
 
     const uint64_t e0 = chunk * kChunk;
@@ -347,7 +337,7 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
     if (chunk == 0 && lo != 0) ok = false;
     if (chunk == num_chunks - 1 && hi != src_bytes) ok = false;
     if (!ok) {
-        if (lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+        if (lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
         return;
     }
 
@@ -379,10 +369,10 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
         row[0] = make_uint4(q.x, __funnelshift_r(q.x, q.y, 16), q.y, __funnelshift_r(q.y, q.z, 16));
         row[1] = make_uint4(q.z, __funnelshift_r(q.z, q.w, 16), q.w, __funnelshift_r(q.w, nxt, 16));
     }
-    if (PREFETCH && CDMA_DEC16_PREFETCH != 0) {
-        // ask L2 for the payload of the chunk a CTA CDMA_DEC16_PREFETCH blocks later will expand
+    if (PREFETCH) {
+        // ask L2 for the payload of the chunk a CTA kDec16PrefetchCtas blocks later will expand
         // (blocks are dispatched in index order; every line still comes from DRAM once)
-        const uint64_t cf = chunk + static_cast<uint64_t>(CDMA_DEC16_PREFETCH) * kDec16Warps;
+        const uint64_t cf = chunk + static_cast<uint64_t>(kDec16PrefetchCtas) * kDec16Warps;
         if (cf < num_chunks) {
             const uint64_t flo = __ldg(table + cf);
             const uint64_t fhi = __ldg(table + cf + 1);
@@ -431,14 +421,14 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
         }
     }
     if (!bad && p != end) bad = true;
-    if (bad && lane == 0) report_status(ws, CDMA_ERR_CORRUPT_STREAM);
+    if (bad && lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
 }
 
 }  // namespace
 
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
-                                  cudaStream_t stream, bool src_on_device) {
+                                  const LaunchCtl& ctl, cudaStream_t stream, bool src_on_device) {
     const uint64_t chunks = num_chunks_of(n);
     if (chunks == 0) return cudaSuccess;
     const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
@@ -448,7 +438,7 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
         const bool prefetch = src_on_device && src_bytes >= (n * 4) / 5;
         auto kernel = prefetch ? zvc_decompress_kernel<uint32_t, true> : zvc_decompress_kernel<uint32_t, false>;
         kernel<<<grid, kDecThreads, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes, d_table, n,
-                                                 static_cast<uint32_t*>(d_dst), d_ws, chunks);
+                                                 static_cast<uint32_t*>(d_dst), d_ws, ctl, chunks);
     } else {
         const dim3 grid16(static_cast<unsigned>((chunks + kDec16Warps - 1) / kDec16Warps));
         // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
@@ -456,7 +446,7 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
         auto kernel = prefetch ? zvc_decompress_kernel_u16<true> : zvc_decompress_kernel_u16<false>;
         kernel<<<grid16, 32 * kDec16Warps, 0, stream>>>(
             static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint16_t*>(d_dst),
-            d_ws, chunks);
+            d_ws, ctl, chunks);
     }
     timing_after_launch(stream);
     count_kernel_launch();

@@ -1,8 +1,9 @@
 """GPU parity at the benchmark's full sizes, in the launch configuration the
 benchmark times.  The whole payload and table are compared with the CPU oracle
-(run on all host cores) where that takes seconds; for the 2^29-element tensors
-the size is checked against the closed form, the round trip bit for bit, and
-sampled chunks byte for byte against the oracle."""
+(run on all host cores), the 2^29-element tensors and the 13-tensor offload set
+included; sizes are also checked against the closed form and every round trip
+bit for bit."""
+import ctypes
 import os
 
 import numpy as np
@@ -87,15 +88,78 @@ def test_config5_large_extremes(which):
     assert codec.decompress(out, c) == n * s
     assert torch.equal(bits(out), bits(x))
     assert codec.canaries_intact()
-    # sampled chunks, byte for byte against the oracle
-    rng = np.random.default_rng(5)
-    k_total = n // 1024
-    picks = sorted(set([0, 1, k_total - 1, k_total // 2] + list(rng.integers(0, k_total, 60))))
-    for k in picks:
-        part = raw_numpy(x.view(-1)[k * 1024:(k + 1) * 1024])
-        want, _ = zvc_c.compress(part)
-        lo, hi = int(table[k]), int(table[k + 1])
-        assert hi - lo == len(want)
-        assert codec.payload[lo:hi].cpu().numpy().tobytes() == want.tobytes()
-    del codec, out, x
+    del out
+    # the whole stream and table, byte for byte against the oracle (all host cores)
+    want, want_table = zvc_c.compress(raw_numpy(x), threads=CORES)
+    assert c == len(want)
+    assert np.array_equal(table, want_table)
+    step = 1 << 28                                           # compare in pieces: bounded host copies
+    for lo in range(0, c, step):
+        hi = min(c, lo + step)
+        assert codec.payload[lo:hi].cpu().numpy().tobytes() == want[lo:hi].tobytes()
+    del want, want_table
+    del codec, x
     torch.cuda.empty_cache()
+
+
+def _ticket_bytes(ctx, ticket):
+    st, c, n = B.cdma_ticket_info(ctx, ticket)
+    assert st == 0
+    st, hp, ht = B.cdma_ticket_host_view(ctx, ticket)
+    assert st == 0
+    payload = np.ctypeslib.as_array((ctypes.c_uint8 * c).from_address(hp)) if c else np.zeros(0, np.uint8)
+    table = np.ctypeslib.as_array((ctypes.c_uint64 * (n // 1024 + 1)).from_address(ht))
+    return c, payload, table
+
+
+@pytest.mark.parametrize("mode", ["staged", "direct", "async"])
+def test_config3_offload_set_full_size(mode):
+    """The 13 conv outputs of the VGG-16-shaped network at batch 64 (3.47 GB): every tensor offloaded
+    (OFF in forward order), each ticket's bytes in the pinned pool compared with the oracle, then
+    prefetched in reverse order (PRE in backward order) and compared bit for bit."""
+    tensors = [t for t, _ in wl.vgg16_offload_set(device="cuda")]
+    assert len(tensors) == 13 and sum(t.numel() for t in tensors) == 867_041_280
+    worst = max(B.cdma_zvc_max_compressed_bytes(t.numel(), B.F32) + 8 * B.cdma_zvc_table_entries(t.numel())
+                + B.cdma_zvc_workspace_bytes(t.numel(), B.F32) + 4096 for t in tensors)
+    pinned = sum(B.cdma_zvc_max_compressed_bytes(t.numel(), B.F32) // 2 + 8 * B.cdma_zvc_table_entries(t.numel())
+                 + 4096 for t in tensors) + worst
+    ctx = B.cdma_ctx_create(pinned, 2 * worst)
+    stream = torch.cuda.Stream()
+    try:
+        tickets = []
+        with torch.cuda.stream(stream):
+            for t in tensors:
+                if mode == "async":
+                    st, tk = B.cdma_offload_async(ctx, t.data_ptr(), t.numel(), B.F32, B.NCHW, stream.cuda_stream)
+                    assert st == 0, B.status_string(st)
+                else:
+                    off = B.cdma_offload if mode == "staged" else B.cdma_offload_direct
+                    c, tk = off(ctx, t.data_ptr(), t.numel(), B.F32, B.NCHW, stream.cuda_stream)
+                    assert c > 0, B.status_string(c)
+                tickets.append(tk)
+            assert B.cdma_ctx_synchronize(ctx) == 0
+            total = 0
+            for t, tk in zip(tensors, tickets):
+                c, payload, table = _ticket_bytes(ctx, tk)
+                want, want_table = zvc_c.compress(raw_numpy(t), threads=CORES)
+                assert c == len(want)
+                assert payload.tobytes() == want.tobytes()
+                assert np.array_equal(table, want_table)
+                total += c
+            assert 2.0 < sum(t.numel() * 4 for t in tensors) / total < 2.6     # size-weighted ratio
+            outs = [torch.empty_like(t) for t in tensors]
+            for i in reversed(range(len(tensors))):
+                if mode == "direct":
+                    r = B.cdma_prefetch_direct(ctx, tickets[i], outs[i].data_ptr(), stream.cuda_stream)
+                    assert r == tensors[i].numel() * 4, B.status_string(r)
+                else:
+                    st = B.cdma_prefetch_async(ctx, tickets[i], outs[i].data_ptr(), stream.cuda_stream)
+                    assert st == 0, B.status_string(st)
+            assert B.cdma_ctx_synchronize(ctx) == 0
+        stream.synchronize()
+        for t, o in zip(tensors, outs):
+            assert torch.equal(bits(o), bits(t))
+    finally:
+        B.cdma_ctx_destroy(ctx)
+        del tensors
+        torch.cuda.empty_cache()

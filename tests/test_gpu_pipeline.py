@@ -196,3 +196,85 @@ def test_direct_offload_writes_the_oracle_stream_into_the_pinned_pool(dtype):
         assert B.cdma_ctx_synchronize(ctx) == 0
     finally:
         B.cdma_ctx_destroy(ctx)
+
+
+def test_offload_async_returns_before_the_compute_stream_has_caught_up():
+    """OFF must not make the host wait for the layer that produces the map (Fig. 2b): with a long-running
+    operation queued on the compute stream in front of it, the call comes back while that operation is
+    still running; the ticket later yields the oracle's bytes."""
+    t = wl.correlated_relu((8, 32, 56, 56), 0.3, seed=77, device="cuda")
+    n = t.numel()
+    ctx = make_ctx([t], slack=1 << 20)
+    stream = torch.cuda.Stream()
+    a = torch.randn(8192, 8192, device="cuda")
+    busy = torch.cuda.Event()
+    try:
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            for _ in range(40):                              # tens of milliseconds of work in front of the offload
+                a = torch.mm(a, a).clamp_(-1.0, 1.0)
+            busy.record(stream)
+            st, ticket = B.cdma_offload_async(ctx, t.data_ptr(), n, B.F32, B.NCHW, stream.cuda_stream)
+            still_running = not busy.query()                 # looked at right after the call returned
+        assert st == 0, B.status_string(st)
+        assert still_running, "cdma_offload_async waited for the compute stream"
+        want, want_table = zvc_c.compress(raw_numpy(t))
+        st, c, n_back = B.cdma_ticket_info(ctx, ticket)      # settles the ticket (waits for its bytes)
+        assert (st, c, n_back) == (0, len(want), n)
+        got, got_table = host_view(ctx, ticket, c, B.cdma_zvc_table_entries(n))
+        assert got.tobytes() == want.tobytes()
+        assert np.array_equal(got_table, want_table)
+        out = torch.zeros_like(t)
+        assert B.cdma_prefetch(ctx, ticket, out.data_ptr(), stream.cuda_stream) == 4 * n
+        assert torch.equal(bits(out), bits(t))
+        assert B.cdma_ctx_synchronize(ctx) == 0
+    finally:
+        B.cdma_ctx_destroy(ctx)
+
+
+def test_offload_async_reports_a_slot_too_small_through_synchronize():
+    t = wl.iid_relu_like((64 * 1024,), 0.9, seed=3, device="cuda")
+    ctx = B.cdma_ctx_create(1 << 20, 2 * 65536)             # staging slot smaller than the payload
+    try:
+        st, ticket = B.cdma_offload_async(ctx, t.data_ptr(), t.numel(), B.F32, B.NCHW, 0)
+        assert st == 0
+        assert B.cdma_ctx_synchronize(ctx) == B.ERR_BUFFER_TOO_SMALL
+        assert B.cdma_ticket_info(ctx, ticket)[0] == B.ERR_BAD_TICKET      # the ticket was dropped
+        assert B.cdma_ctx_synchronize(ctx) == 0
+        s = wl.iid_relu_like((8 * 1024,), 0.1, seed=4, device="cuda")      # the context still works
+        st, ticket = B.cdma_offload_async(ctx, s.data_ptr(), s.numel(), B.F32, B.NCHW, 0)
+        assert st == 0
+        out = torch.zeros_like(s)
+        assert B.cdma_prefetch(ctx, ticket, out.data_ptr(), 0) == 4 * s.numel()
+        assert torch.equal(bits(out), bits(s))
+    finally:
+        B.cdma_ctx_destroy(ctx)
+
+
+def test_prefetch_async_then_direct_offload_into_the_recycled_region():
+    """The end of a backward pass followed by the next forward pass: a prefetch whose host-to-device copy
+    is still in flight gives its pinned region back, and a direct offload (a kernel that writes the pool
+    from the caller's stream) is handed that very region.  Both tensors must come out bit-exact."""
+    a = wl.iid_relu_like((6_000_000,), 0.6, seed=41, device="cuda")      # ~15 MB payload: a copy that takes a while
+    b = wl.iid_relu_like((6_000_000,), 0.6, seed=42, device="cuda")
+    need = B.cdma_zvc_max_compressed_bytes(a.numel(), B.F32) + 8 * B.cdma_zvc_table_entries(a.numel()) + 4096
+    ws = B.cdma_zvc_workspace_bytes(a.numel(), B.F32)
+    ctx = B.cdma_ctx_create(need + 8192, 2 * (need + ws + 4096))          # room for exactly one ticket
+    stream = torch.cuda.Stream()
+    try:
+        for _ in range(4):
+            c, tk_a = B.cdma_offload_direct(ctx, a.data_ptr(), a.numel(), B.F32, B.NCHW, stream.cuda_stream)
+            assert c > 0, B.status_string(c)
+            out_a = torch.zeros_like(a)
+            assert B.cdma_prefetch_async(ctx, tk_a, out_a.data_ptr(), stream.cuda_stream) == 0
+            # no synchronisation here: the copy of a's payload out of the pool may still be running
+            c, tk_b = B.cdma_offload_direct(ctx, b.data_ptr(), b.numel(), B.F32, B.NCHW, stream.cuda_stream)
+            assert c > 0, B.status_string(c)
+            out_b = torch.zeros_like(b)
+            assert B.cdma_prefetch(ctx, tk_b, out_b.data_ptr(), stream.cuda_stream) == 4 * b.numel()
+            assert B.cdma_ctx_synchronize(ctx) == 0
+            stream.synchronize()
+            assert torch.equal(bits(out_a), bits(a))
+            assert torch.equal(bits(out_b), bits(b))
+    finally:
+        B.cdma_ctx_destroy(ctx)

@@ -199,9 +199,10 @@ def sentinel(j, s):
 
 
 @pytest.mark.parametrize("s", [4, 2])
-def test_every_pattern_up_to_12_elements(s):
+def test_every_pattern_of_tiny_inputs(s):
+    # every zero / non-zero pattern of every length up to 16 (4-byte elements; up to 12 for 2-byte ones)
     it = np.uint32 if s == 4 else np.uint16
-    for n in range(1, 13):
+    for n in range(1, 17 if s == 4 else 13):
         for bits in itertools.product([False, True], repeat=n):
             x = np.array([sentinel(j, s) if b else 0 for j, b in enumerate(bits)], dtype=it)
             payload, _ = zvc_c.compress(x)

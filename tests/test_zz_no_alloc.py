@@ -1,9 +1,10 @@
 """GPU: the compression entry point for callers that cannot allocate device
 memory (cdma_zvc_compress_static_ws) must produce exactly what the ordinary
 entry point produces -- same return value, same payload bytes, same offset
-table (integer/byte work: tolerance 0) -- on two calls in a row, the second of
-which would be wrong if the first call's leftovers in the shared built-in
-workspace were not cleared.
+table (integer/byte work: tolerance 0), which are also the CPU oracle's -- on two
+calls in a row, the second of which would be wrong if the first call's leftovers
+in the shared built-in workspace were mistaken for its own.  The calls must also
+leave the amount of free device memory unchanged.
 
 This file is named to be collected last: a run that stops at the first failure
 has then already run every other test.  It passes on its own in a fresh process
@@ -13,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import zvc_c
 from paper_1705_01626_b200 import binding as B
 from paper_1705_01626_b200 import workloads as wl
 
@@ -33,28 +35,54 @@ def compress_both_ways(x, stream=0):
     assert c_ref >= 0, B.status_string(c_ref)
     payload = torch.full((cap,), 0xEE, dtype=torch.uint8, device="cuda")
     table = torch.full((entries,), -1, dtype=torch.int64, device="cuda")
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     c = B.cdma_zvc_compress_static_ws(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
                                       stream)
+    free_after = torch.cuda.mem_get_info()[0]
     assert c == c_ref, (c, c_ref, B.status_string(c))
     assert torch.equal(payload[:c], ref_payload[:c])
     assert torch.equal(table, ref_table)
-    return c
+    it = torch.int32 if x.element_size() == 4 else torch.int16
+    raw = x.contiguous().view(-1).view(it).cpu().numpy().view(np.uint32 if x.element_size() == 4 else np.uint16)
+    want, want_table = zvc_c.compress(raw)
+    assert c == len(want) and payload[:c].cpu().numpy().tobytes() == want.tobytes()
+    assert np.array_equal(table.cpu().numpy().view(np.uint64), want_table)
+    return c, free_before - free_after
 
 
 def test_two_calls_in_a_row_match_the_ordinary_entry_point():
     # first a large, dense-ish tensor (many tiles, large offsets left behind in the workspace) ...
     big = wl.iid_relu_like((3_000_000 + 123,), 0.8, seed=wl.seed_for(7, 0), device="cuda")
-    c1 = compress_both_ways(big)
+    # (the very first call on a device loads the module that holds the built-in workspace, which is when
+    # its memory is taken: warm up once, as a caller on an eviction path would at start-up)
+    assert B.cdma_zvc_compress_static_ws(0, 0, B.F32, B.NCHW, 0, 0, torch.zeros(1, dtype=torch.int64,
+                                         device="cuda").data_ptr(), 0) == 0
+    c1, used1 = compress_both_ways(big)
     # ... then a smaller, sparser one that reuses the first tiles' descriptors
     small = wl.correlated_relu((4, 16, 56, 56), 0.2, seed=wl.seed_for(7, 1), device="cuda")
-    c2 = compress_both_ways(small)
+    c2, used2 = compress_both_ways(small)
     assert c2 < c1
+    assert used1 == 0 and used2 == 0                          # the calls took no device memory
     # and once more on a side stream with 2-byte elements
     half = wl.iid_relu_like((500_000 + 7,), 0.3, seed=wl.seed_for(7, 2), device="cuda", dtype=torch.float16,
                             floor=2.0 ** -10)
     s = torch.cuda.Stream()
     torch.cuda.synchronize()
     compress_both_ways(half, s.cuda_stream)
+
+
+def test_a_source_in_page_locked_host_memory_is_read_over_the_link():
+    n = 200_000 + 9
+    h = wl.iid_relu_like((n,), 0.3, seed=wl.seed_for(7, 3), device="cpu").pin_memory()
+    cap = B.cdma_zvc_max_compressed_bytes(n, B.F32)
+    payload = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    table = torch.zeros(B.cdma_zvc_table_entries(n), dtype=torch.int64, device="cuda")
+    c = B.cdma_zvc_compress_static_ws(h.data_ptr(), n, B.F32, B.NCHW, payload.data_ptr(), cap, table.data_ptr(), 0)
+    want, want_table = zvc_c.compress(h.numpy().view(np.uint32))
+    assert c == len(want), B.status_string(c)
+    assert payload[:c].cpu().numpy().tobytes() == want.tobytes()
+    assert np.array_equal(table.cpu().numpy().view(np.uint64), want_table)
 
 
 def test_sizes_beyond_the_built_in_workspace_are_refused():
