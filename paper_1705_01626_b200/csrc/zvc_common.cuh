@@ -134,6 +134,10 @@ __device__ inline void report_decode_error(uint64_t* ws, const LaunchCtl& ctl, u
 cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst,
                                 uint64_t cap, uint64_t* d_table, uint64_t* d_ws, const LaunchCtl& ctl,
                                 cudaStream_t stream, bool src_on_device = true);
+// The kernel for device-resident 2-byte tensors of at least one tile (zvc_compress_rows.cu).
+bool zvc_compress_rows_usable(const void* d_src, uint64_t n, uint32_t elem_size);
+cudaError_t launch_zvc_compress_rows(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
+                                     uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream);
 cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
                                      void* d_relu_out, void* d_dst, uint64_t cap, uint64_t* d_table,
                                      uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream,
