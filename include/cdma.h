@@ -225,6 +225,36 @@ int cdma_zvc_decompress_async(const void* d_src, uint64_t src_bytes,
                               uint64_t workspace_bytes, void* cuda_stream,
                               uint64_t* h_result);
 
+/*
+ * Backward pass of the activation function straight from the compressed map.
+ * The offloaded maps are needed again in the backward pass (Section II-B); for a
+ * ReLU layer all that is needed of y = max(x, 0) is which elements are non-zero,
+ * and that is what the masks of the stream record (Section V-A).  The call
+ * computes dx = dy where the element of the compressed tensor is non-zero, else
+ * +0, reading the masks only: the dense y is never rebuilt in memory (Section IX
+ * leaves keeping activations compressed as future work).
+ *
+ *   d_src, src_bytes, d_table   payload, its exact size and offset table, as for
+ *                               cdma_zvc_decompress (validated the same way)
+ *   d_dy        incoming gradient, n*s bytes, 16-byte aligned, same dtype
+ *   d_dx        outgoing gradient, n*s bytes, 16-byte aligned; may be d_dy itself
+ *               (in place), must not overlap it otherwise, nor the payload
+ *   d_workspace >= cdma_zvc_workspace_bytes(n, dtype)
+ *
+ * For a payload produced from a ReLU output (cdma_zvc_relu_compress or
+ * compression of y) this is the framework's ReLU backward, bit for bit: elements
+ * whose y is a NaN pass dy on, as a comparison "y <= 0 ? 0 : dy" does.
+ * cdma_zvc_relu_backward waits for the stream and returns n*s or -status;
+ * the _async form only enqueues, h_result as for cdma_zvc_decompress_async.
+ */
+int64_t cdma_zvc_relu_backward(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
+                               uint64_t n, int dtype, int layout, const void* d_dy, void* d_dx,
+                               void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
+int cdma_zvc_relu_backward_async(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
+                                 uint64_t n, int dtype, int layout, const void* d_dy, void* d_dx,
+                                 void* d_workspace, uint64_t workspace_bytes, void* cuda_stream,
+                                 uint64_t* h_result);
+
 /* ------------------------------------------------------------------------ *
  * Run-length comparison codec (Section V-A, "Run-length encoding compression";
  * its dependence on the activation layout is the subject of Section VI-A,

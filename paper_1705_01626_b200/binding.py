@@ -63,6 +63,10 @@ _SIGNATURES = {
                                       c_void_p, c_uint64, c_void_p]),
     "cdma_zvc_decompress_async": (c_int, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p,
                                           c_void_p, c_uint64, c_void_p, c_void_p]),
+    "cdma_zvc_relu_backward": (c_int64, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p, c_void_p,
+                                         c_void_p, c_uint64, c_void_p]),
+    "cdma_zvc_relu_backward_async": (c_int, [c_void_p, c_uint64, c_void_p, c_uint64, c_int, c_int, c_void_p, c_void_p,
+                                             c_void_p, c_uint64, c_void_p, c_void_p]),
     "cdma_rle_compress": (c_int64, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64, c_void_p,
                                     c_void_p, c_uint64, c_void_p]),
     "cdma_rle_compress_async": (c_int, [c_void_p, c_uint64, c_int, c_int, c_void_p, c_uint64, c_void_p,
@@ -216,6 +220,21 @@ def cdma_zvc_decompress_async(d_src, src_bytes, d_table, n, dtype, layout, d_dst
     return int(lib().cdma_zvc_decompress_async(_vp(d_src), src_bytes, _vp(d_table), n, dtype, layout,
                                                _vp(d_dst), _vp(d_workspace), workspace_bytes,
                                                _vp(cuda_stream), _vp(h_result)))
+
+
+def cdma_zvc_relu_backward(d_src, src_bytes, d_table, n, dtype, layout, d_dy, d_dx, d_workspace, workspace_bytes,
+                           cuda_stream=0) -> int:
+    """dx = dy where the compressed tensor's element is non-zero, else 0, from the masks alone.
+    Returns n*s, or a negative status."""
+    return int(lib().cdma_zvc_relu_backward(_vp(d_src), src_bytes, _vp(d_table), n, dtype, layout, _vp(d_dy), _vp(d_dx),
+                                            _vp(d_workspace), workspace_bytes, _vp(cuda_stream)))
+
+
+def cdma_zvc_relu_backward_async(d_src, src_bytes, d_table, n, dtype, layout, d_dy, d_dx, d_workspace, workspace_bytes,
+                                 cuda_stream, h_result) -> int:
+    return int(lib().cdma_zvc_relu_backward_async(_vp(d_src), src_bytes, _vp(d_table), n, dtype, layout, _vp(d_dy),
+                                                  _vp(d_dx), _vp(d_workspace), workspace_bytes, _vp(cuda_stream),
+                                                  _vp(h_result)))
 
 
 def cdma_ctx_create(pinned_bytes: int, device_staging_bytes: int):

@@ -290,6 +290,46 @@ int64_t cdma_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_
     return static_cast<int64_t>(n) * cdma_dtype_size(dtype);
 }
 
+// ---- backward pass of the activation function from the compressed map ----------------
+
+int cdma_zvc_relu_backward_async(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                 int dtype, int layout, const void* d_dy, void* d_dx, void* d_workspace,
+                                 uint64_t workspace_bytes, void* cuda_stream, uint64_t* h_result) {
+    const int st = check_common(n, dtype, layout, d_dx, d_src, d_table, d_workspace, workspace_bytes);
+    if (st != CDMA_OK) return st;
+    if ((src_bytes != 0 && d_src == nullptr) || (n != 0 && d_dy == nullptr) || h_result == nullptr)
+        return CDMA_ERR_INVALID_ARG;
+    if (!aligned(d_dy, 16)) return CDMA_ERR_ALIGNMENT;
+    const uint32_t s = cdma_dtype_size(dtype);
+    // dx may be dy itself (in place); any other overlap, or one with the payload, is refused
+    if (overlaps(d_dx, n * s, d_src, src_bytes) || overlaps(d_dy, n * s, d_src, src_bytes)) return CDMA_ERR_INVALID_ARG;
+    if (d_dx != d_dy && overlaps(d_dx, n * s, d_dy, n * s)) return CDMA_ERR_INVALID_ARG;
+    const uint64_t windows = (n + kWindow - 1) / kWindow;
+    if (src_bytes < 4 * windows || src_bytes > 4 * windows + static_cast<uint64_t>(s) * n || src_bytes % s != 0)
+        return CDMA_ERR_CORRUPT_STREAM;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint64_t* ws = static_cast<uint64_t*>(d_workspace);
+    if (n == 0) return result_without_kernel(ws, 0, h_result, stream) == cudaSuccess ? CDMA_OK : CDMA_ERR_CUDA;
+    const LaunchCtl ctl = make_launch_ctl(h_result);
+    if (launch_zvc_relu_backward(d_src, src_bytes, d_table, n, s, d_dy, d_dx, ws, ctl, stream) != cudaSuccess)
+        return CDMA_ERR_CUDA;
+    if (finish_result(ws, ctl, h_result, stream) != cudaSuccess) return CDMA_ERR_CUDA;
+    return CDMA_OK;
+}
+
+int64_t cdma_zvc_relu_backward(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n, int dtype,
+                               int layout, const void* d_dy, void* d_dx, void* d_workspace, uint64_t workspace_bytes,
+                               void* cuda_stream) {
+    uint64_t result[2] = {0, 0};
+    const int st = cdma_zvc_relu_backward_async(d_src, src_bytes, d_table, n, dtype, layout, d_dy, d_dx, d_workspace,
+                                                workspace_bytes, cuda_stream, result);
+    if (st != CDMA_OK) return -static_cast<int64_t>(st);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return -static_cast<int64_t>(CDMA_ERR_CUDA);
+    if (result[1] != 0) return -static_cast<int64_t>(result[1]);
+    return static_cast<int64_t>(n) * cdma_dtype_size(dtype);
+}
+
 // ---- run-length comparison codec (4-byte elements) -----------------------------------
 
 int cdma_rle_compress_async(const void* d_src, uint64_t n, int dtype, int layout, void* d_dst,

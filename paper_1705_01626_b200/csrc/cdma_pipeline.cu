@@ -315,6 +315,13 @@ int cdma_ctx_create(uint64_t pinned_bytes, uint64_t device_staging_bytes, cdma_c
         if (cudaEventCreateWithFlags(&ctx->pool_read, cudaEventDisableTiming) != cudaSuccess) {
             st = CDMA_ERR_CUDA; break;
         }
+        // cdma_offload_async must not make the host wait: no kernel is loaded lazily at its first launch
+        cdma::preload_compress_kernels();
+        {
+            cudaFuncAttributes attr;
+            (void)cudaFuncGetAttributes(&attr, offload_copy_kernel);
+            (void)cudaGetLastError();
+        }
         for (uint32_t i = 0; i < kSlots && st == CDMA_OK; ++i) {
             ctx->slots[i].base = ctx->d_staging ? ctx->d_staging + i * slot_bytes : nullptr;
             ctx->slots[i].bytes = slot_bytes;

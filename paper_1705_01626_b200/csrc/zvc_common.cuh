@@ -138,6 +138,8 @@ cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_siz
 bool zvc_compress_rows_usable(const void* d_src, uint64_t n, uint32_t elem_size);
 cudaError_t launch_zvc_compress_rows(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
                                      uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream);
+void preload_compress_rows_kernel();
+void preload_compress_kernels();     // load every compression kernel now rather than at its first launch
 cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
                                      void* d_relu_out, void* d_dst, uint64_t cap, uint64_t* d_table,
                                      uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream,
@@ -145,6 +147,9 @@ cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t ele
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
                                   const LaunchCtl& ctl, cudaStream_t stream, bool src_on_device = true);
+cudaError_t launch_zvc_relu_backward(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                     uint32_t elem_size, const void* d_dy, void* d_dx, uint64_t* d_ws,
+                                     const LaunchCtl& ctl, cudaStream_t stream);
 cudaError_t launch_rle_compress(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
                                 uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream);
 cudaError_t launch_rle_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,

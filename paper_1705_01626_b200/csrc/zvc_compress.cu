@@ -513,6 +513,16 @@ cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_siz
     return e;
 }
 
+// With lazy module loading the first launch of a kernel in a process can wait for the device
+// to go idle; a context that promises not to make the host wait loads its kernels up front.
+void preload_compress_kernels() {
+    cudaFuncAttributes a;
+    (void)cudaFuncGetAttributes(&a, zvc_compress_kernel<uint32_t, false>);
+    (void)cudaFuncGetAttributes(&a, zvc_compress_kernel_u16<false>);
+    preload_compress_rows_kernel();
+    (void)cudaGetLastError();
+}
+
 cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
                                      void* d_relu_out, void* d_dst, uint64_t cap, uint64_t* d_table,
                                      uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream,

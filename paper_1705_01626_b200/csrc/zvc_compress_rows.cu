@@ -256,6 +256,12 @@ EncodeTiledFn encode_tiled() {
 
 }  // namespace
 
+void preload_compress_rows_kernel() {
+    cudaFuncAttributes a;
+    (void)cudaFuncGetAttributes(&a, zvc_compress_rows_kernel_u16);
+    (void)encode_tiled();
+}
+
 bool zvc_compress_rows_usable(const void* d_src, uint64_t n, uint32_t elem_size) {
     // 2-byte elements, at least one whole tile, rows addressable with 32-bit coordinates, and an
     // encoder to describe them

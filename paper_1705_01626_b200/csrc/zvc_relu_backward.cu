@@ -1,0 +1,162 @@
+// Backward pass of the activation function straight from the compressed map.
+//
+// The offloaded activation maps are needed again in the backward pass (Section
+// II-B), and for a ReLU layer all the backward pass needs of y = max(x, 0) is which
+// elements are non-zero: dx = dy where y != 0, else 0.  That is exactly what the
+// masks of the compressed stream say (Section V-A: bit i of a window's mask is set
+// when element i is non-zero), so the dense y never has to be rebuilt in memory
+// (the direction Section IX leaves as future work: keeping activations compressed).
+// The kernel walks the masks of the payload, reads dy, writes dx: 2 n s + C bytes of
+// traffic instead of the 4 n s + C of decompressing y and then running the
+// framework's backward kernel over y and dy.
+//
+// One warp per chunk.  The chunk's payload lines are first pulled into L1 by one
+// load per lane, all in flight together; the self-delimiting walk from mask to mask
+// (Section V-A) then runs on L1 hits, every lane following it and lane w keeping the
+// mask of window w.  A lane then gates 16 bytes of dy per round (4 or 8 elements)
+// with its bits of its window's mask, fetched by one shuffle.  The table and the walk
+// are validated as in decompression: offsets inside the payload, the walk ending
+// exactly at the chunk's end, no mask bit naming an element at index >= n.
+#include "zvc_common.cuh"
+
+namespace cdma {
+
+namespace {
+
+constexpr uint32_t kBwdWarps = 8;
+
+__device__ __forceinline__ uint32_t ld_mask(const uint8_t* p, uint32_t elem_size) {
+    // a mask starts on an element boundary: 4-byte aligned for 4-byte elements, 2-byte aligned otherwise
+    if (elem_size == 4) return __ldg(reinterpret_cast<const uint32_t*>(p));
+    const uint32_t lo = __ldg(reinterpret_cast<const uint16_t*>(p));
+    const uint32_t hi = __ldg(reinterpret_cast<const uint16_t*>(p + 2));
+    return lo | (hi << 16);
+}
+
+template <uint32_t S>
+__global__ void __launch_bounds__(32 * kBwdWarps)
+zvc_relu_backward_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, const uint64_t* __restrict__ table,
+                         uint64_t n, const uint8_t* __restrict__ dy, uint8_t* __restrict__ dx,
+                         uint64_t* __restrict__ ws, const LaunchCtl ctl, uint64_t num_chunks) {
+    constexpr uint32_t EPL = 16 / S;                 // elements a lane gates per round (one 16-byte vector)
+    constexpr uint32_t LPW = kWindow / EPL;          // lanes per window
+    constexpr uint32_t WPR = 32 / LPW;               // windows per round
+    const uint32_t lane = lane_id();
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * kBwdWarps + warp;
+    if (blockIdx.x == 0 && threadIdx.x == 0) init_decode_result(ws, ctl, n * S);
+    if (chunk >= num_chunks) return;
+
+    const uint64_t e0 = chunk * kChunk;
+    const uint32_t nelem = (n - e0 < kChunk) ? static_cast<uint32_t>(n - e0) : kChunk;
+    const uint32_t nwin = (nelem + kWindow - 1) / kWindow;
+
+    // ---- the chunk's byte range, validated -------------------------------------------------------
+    const uint64_t lo = __ldg(table + chunk);
+    const uint64_t hi = __ldg(table + chunk + 1);
+    bool ok = (lo <= hi) && (hi <= src_bytes) && (hi - lo >= 4ull * nwin) &&
+              (hi - lo <= 4ull * nwin + static_cast<uint64_t>(S) * nelem) && (lo % S == 0) && ((hi - lo) % S == 0);
+    if (chunk == 0 && lo != 0) ok = false;
+    if (chunk == num_chunks - 1 && hi != src_bytes) ok = false;
+    if (!ok) {
+        if (lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
+        return;
+    }
+
+    // ---- bring the chunk's payload lines (at most 34) close: one load per lane, a second for the first lanes --
+    {
+        const uint64_t line0 = lo & ~127ull;
+        uint32_t sink = 0;
+        for (uint64_t a = line0 + 128ull * lane; a < hi; a += 128ull * 32) {
+            // any word of the line that lies inside the payload
+            const uint64_t at = a < lo ? lo : a;
+            uint32_t v;
+            asm volatile("ld.global.ca.u16 %0, [%1];" : "=r"(v) : "l"(src + at) : "memory");
+            sink ^= v;
+        }
+        if (sink == 0x9e3779b9u) asm volatile("" ::: "memory");     // keeps the loads; never true for 16-bit values
+    }
+
+    // ---- the walk: lane w ends up with the mask of window w ----------------------------------------
+    uint64_t p = lo;
+    uint32_t mine = 0;
+    bool bad = false;
+    for (uint32_t w = 0; w < nwin; ++w) {
+        if (p + 4 > hi) { bad = true; break; }
+        const uint32_t m = ld_mask(src + p, S);
+        if (lane == w) mine = m;
+        p += 4ull + static_cast<uint64_t>(S) * __popc(m);
+    }
+    if (!bad && p != hi) bad = true;
+    // a short last window must not name elements beyond n
+    if (!bad && nelem != kChunk) {
+        const uint32_t tail = nelem & 31u;
+        const uint32_t last_mask = __shfl_sync(0xffffffffu, mine, nwin - 1);
+        if (tail != 0 && (last_mask >> tail) != 0) bad = true;
+    }
+    if (bad) {
+        if (lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
+        return;
+    }
+
+    // ---- gate dy with the masks ----------------------------------------------------------------------
+    if (nelem == kChunk) {
+        const uint4* in = reinterpret_cast<const uint4*>(dy + e0 * S) + lane;
+        uint4* out = reinterpret_cast<uint4*>(dx + e0 * S) + lane;
+        const uint32_t sh = EPL * (lane % LPW);
+#pragma unroll
+        for (uint32_t r = 0; r < kChunkWindows / WPR; ++r) {
+            const uint32_t m = __shfl_sync(0xffffffffu, mine, r * WPR + lane / LPW);
+            const uint32_t bits = m >> sh;
+            uint4 v = __ldcs(in + 32 * r);
+            if (S == 4) {
+                v.x = (bits & 1u) ? v.x : 0u;
+                v.y = (bits & 2u) ? v.y : 0u;
+                v.z = (bits & 4u) ? v.z : 0u;
+                v.w = (bits & 8u) ? v.w : 0u;
+            } else {
+                // two elements per word: keep masks from two bits each
+                v.x &= ((bits & 1u) ? 0xffffu : 0u) | ((bits & 2u) ? 0xffff0000u : 0u);
+                v.y &= ((bits & 4u) ? 0xffffu : 0u) | ((bits & 8u) ? 0xffff0000u : 0u);
+                v.z &= ((bits & 16u) ? 0xffffu : 0u) | ((bits & 32u) ? 0xffff0000u : 0u);
+                v.w &= ((bits & 64u) ? 0xffffu : 0u) | ((bits & 128u) ? 0xffff0000u : 0u);
+            }
+            __stcs(out + 32 * r, v);
+        }
+    } else {
+        // ragged last chunk: lane = element, one window per step
+        for (uint32_t w = 0; w < nwin; ++w) {
+            const uint32_t m = __shfl_sync(0xffffffffu, mine, w);
+            const uint64_t j = e0 + w * kWindow + lane;
+            if (j < n) {
+                const bool keep = (m >> lane) & 1u;
+                if (S == 4) reinterpret_cast<uint32_t*>(dx)[j] = keep ? reinterpret_cast<const uint32_t*>(dy)[j] : 0u;
+                else reinterpret_cast<uint16_t*>(dx)[j] = keep ? reinterpret_cast<const uint16_t*>(dy)[j] : uint16_t(0);
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_zvc_relu_backward(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                     uint32_t elem_size, const void* d_dy, void* d_dx, uint64_t* d_ws,
+                                     const LaunchCtl& ctl, cudaStream_t stream) {
+    const uint64_t chunks = num_chunks_of(n);
+    if (chunks == 0) return cudaSuccess;
+    const dim3 grid(static_cast<unsigned>((chunks + kBwdWarps - 1) / kBwdWarps));
+    timing_before_launch(stream);
+    if (elem_size == 4)
+        zvc_relu_backward_kernel<4><<<grid, 32 * kBwdWarps, 0, stream>>>(
+            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<const uint8_t*>(d_dy),
+            static_cast<uint8_t*>(d_dx), d_ws, ctl, chunks);
+    else
+        zvc_relu_backward_kernel<2><<<grid, 32 * kBwdWarps, 0, stream>>>(
+            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<const uint8_t*>(d_dy),
+            static_cast<uint8_t*>(d_dx), d_ws, ctl, chunks);
+    timing_after_launch(stream);
+    count_kernel_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace cdma
