@@ -83,7 +83,7 @@ def closed_form_bytes(n: int, nnz: int, s: int) -> int:
 
 
 def compress(x: np.ndarray, capacity: int | None = None, threads: int = 1):
-    """Compress ``x`` (any dtype of 2 or 4 bytes per element, memory order).
+    """Compress ``x`` (any dtype of 1, 2 or 4 bytes per element, memory order).
 
     Returns ``(payload uint8[C], table uint64[K+1])``.  With ``capacity`` given
     the destination is that many bytes and a too-small one raises

@@ -31,7 +31,9 @@ def _raw(x: np.ndarray) -> np.ndarray:
         return x.view(np.uint32)
     if x.dtype.itemsize == 2:
         return x.view(np.uint16)
-    raise ValueError("elements must be 2 or 4 bytes")
+    if x.dtype.itemsize == 1:
+        return x.view(np.uint8)
+    raise ValueError("elements must be 1, 2 or 4 bytes")
 
 
 def nonzero_bits(x: np.ndarray) -> np.ndarray:
@@ -124,7 +126,7 @@ def split_stream(payload: np.ndarray, n: int, s: int):
     out_masks = np.zeros(w, dtype=np.uint32)
     chunks = []
     pos = 0
-    vt = np.dtype("<u4") if s == 4 else np.dtype("<u2")
+    vt = {4: np.dtype("<u4"), 2: np.dtype("<u2"), 1: np.dtype("u1")}[s]
     for i in range(w):
         if pos + 4 > payload.size:
             raise ValueError("stream ends inside a mask")
@@ -137,4 +139,4 @@ def split_stream(payload: np.ndarray, n: int, s: int):
         chunks.append(payload[pos:pos + s * cnt])
         pos += s * cnt
     vals = np.concatenate(chunks).view(vt) if chunks else np.zeros(0, dtype=vt)
-    return out_masks, vals.astype(np.uint32 if s == 4 else np.uint16), pos
+    return out_masks, vals.astype({4: np.uint32, 2: np.uint16, 1: np.uint8}[s]), pos

@@ -10,7 +10,7 @@
  * What it states (paper Section V-A, "Zero-value compression", and the
  * decompression engine of Section V-B, Fig. 10b):
  *
- *   - The input is n elements of s bytes each (s = 4 or 2), in memory order.
+ *   - The input is n elements of s bytes each (s = 4, 2 or 1), in memory order.
  *   - Elements are grouped into windows of 32 consecutive elements.  For each
  *     window a 32-bit mask is produced: bit i is 1 when element i of the
  *     window is non-zero, 0 when it is zero.  "Zero" means every byte of the
@@ -25,8 +25,10 @@
  * Readings where the paper is silent:
  * bit i (least significant = 0) belongs to element i of the window; the mask
  * is stored least-significant byte first; a short last window has zero bits
- * for the missing elements and no values for them; for 2-byte elements the
- * window is still 32 elements and the mask 32 bits, with no padding.
+ * for the missing elements and no values for them; for 2-byte and 1-byte
+ * elements the window is still 32 elements and the mask 32 bits, with no
+ * padding (the paper's engine is 32-bit only, Section V-B), so the stream of n
+ * elements with nnz non-zero ones is always 4*ceil(n/32) + s*nnz bytes.
  *
  * Framing for parallel decoders (ours, outside the payload): a table of
  * ceil(n/1024)+1 byte offsets, entry k being where the record of window 32k
@@ -127,7 +129,7 @@ int64_t zvc_oracle_compress(const void *src, uint64_t n, unsigned s,
 {
     uint64_t windows, end;
     int overflow = 0;
-    if (s != 2 && s != 4) return -1;
+    if (s != 1 && s != 2 && s != 4) return -1;
     if (n != 0 && src == NULL) return -1;
     if (cap != 0 && dst == NULL) return -1;
     windows = (n + ORACLE_WINDOW - 1) / ORACLE_WINDOW;
@@ -151,7 +153,7 @@ int64_t zvc_oracle_decompress(const void *src, uint64_t src_bytes, uint64_t n,
     const unsigned char *in = (const unsigned char *)src;
     unsigned char *out = (unsigned char *)dst;
     uint64_t windows, w, pos = 0;
-    if (s != 2 && s != 4) return -1;
+    if (s != 1 && s != 2 && s != 4) return -1;
     if (n != 0 && dst == NULL) return -1;
     if (src_bytes != 0 && src == NULL) return -1;
     windows = (n + ORACLE_WINDOW - 1) / ORACLE_WINDOW;
@@ -189,7 +191,7 @@ int zvc_oracle_check_table(const void *src, uint64_t src_bytes, uint64_t n,
 {
     const unsigned char *in = (const unsigned char *)src;
     uint64_t windows, w, pos = 0;
-    if (s != 2 && s != 4) return -1;
+    if (s != 1 && s != 2 && s != 4) return -1;
     if (table == NULL) return -1;
     windows = (n + ORACLE_WINDOW - 1) / ORACLE_WINDOW;
     for (w = 0; w < windows; ++w) {
@@ -247,7 +249,7 @@ int64_t zvc_oracle_compress_mt(const void *src, uint64_t n, unsigned s,
     int pass, overflow = 0;
     mt_job *jobs;
     pthread_t *tids;
-    if (s != 2 && s != 4) return -1;
+    if (s != 1 && s != 2 && s != 4) return -1;
     if (threads == 0) return -1;
     windows = (n + ORACLE_WINDOW - 1) / ORACLE_WINDOW;
     chunks = (windows + ORACLE_CHUNK_WINDOWS - 1) / ORACLE_CHUNK_WINDOWS;
@@ -316,7 +318,7 @@ int64_t zvc_oracle_decompress_mt(const void *src, uint64_t src_bytes,
     int bad = 0;
     mt_djob *jobs;
     pthread_t *tids;
-    if (s != 2 && s != 4) return -1;
+    if (s != 1 && s != 2 && s != 4) return -1;
     if (threads == 0 || table == NULL) return -1;
     chunks = (n + chunk - 1) / chunk;
     if (chunks == 0) return zvc_oracle_decompress(src, src_bytes, n, s, dst);

@@ -24,6 +24,10 @@ def u16(vals):
     return np.array(vals, dtype=np.uint16)
 
 
+def u8(vals):
+    return np.array(vals, dtype=np.uint8)
+
+
 # --------------------------------------------------------------------------- #
 # hand-written byte vectors (typed out, not computed)
 # --------------------------------------------------------------------------- #
@@ -50,6 +54,12 @@ HAND_VECTORS = [
     # fp16, n=34: one value in window 0 makes window 1's mask start at byte 6
     (u16([0] * 7 + [0xBEEF] + [0] * 24 + [0x1234, 0x0000]),
      "80000000" "efbe" "01000000" "3412"),
+    # 1-byte elements (fp8 / int8), n=6: elements 1, 2 (0x80: -0.0 in fp8) and 5 non-zero -> mask 0b100110
+    (u8([0x00, 0x7F, 0x80, 0x00, 0x00, 0x01]),
+     "26000000" "7f" "80" "01"),
+    # 1-byte elements, n=35: three values in window 0 make window 1's mask start at byte 7 (odd address)
+    (u8([0xAA] + [0] * 15 + [0xBB] + [0] * 14 + [0xCC] + [0x00, 0xDD, 0xEE]),
+     "01000180" "aa" "bb" "cc" "06000000" "dd" "ee"),
 ]
 
 
@@ -110,19 +120,19 @@ BOUNDARY_N = [0, 1, 31, 32, 33, 63, 64, 65, 1023, 1024, 1025, 2047, 2048, 2049,
 
 def random_sparse(n, density, seed, dtype):
     rng = np.random.default_rng(seed)
-    it = np.uint32 if np.dtype(dtype).itemsize == 4 else np.uint16
+    it = {4: np.uint32, 2: np.uint16, 1: np.uint8}[np.dtype(dtype).itemsize]
     raw = rng.integers(1, np.iinfo(it).max, size=n, dtype=it, endpoint=True)
     raw[rng.random(n) >= density] = 0
     return raw.view(dtype)
 
 
-@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("dtype", [np.float32, np.float16, np.uint8])
 @pytest.mark.parametrize("n", BOUNDARY_N)
 def test_closed_form_size_and_round_trip(n, dtype):
     s = np.dtype(dtype).itemsize
     for seed in range(3):
         x = random_sparse(n, [0.1, 0.5, 0.9][seed], 100 + seed, dtype)
-        nnz = int(np.count_nonzero(x.view(np.uint32 if s == 4 else np.uint16)))
+        nnz = int(np.count_nonzero(x.view({4: np.uint32, 2: np.uint16, 1: np.uint8}[s])))
         payload, table = zvc_c.compress(x)
         assert len(payload) == 4 * ((n + 31) // 32) + s * nnz
         assert len(payload) == zvc_c.closed_form_bytes(n, nnz, s)
@@ -133,7 +143,7 @@ def test_closed_form_size_and_round_trip(n, dtype):
         assert np.array_equal(zvc_numpy.table(x), table)
 
 
-@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("dtype", [np.float32, np.float16, np.uint8])
 @pytest.mark.parametrize("n", [1, 32, 33, 1024, 1025, 5000])
 def test_all_zero(n, dtype):
     x = np.zeros(n, dtype=dtype)
@@ -147,12 +157,12 @@ def test_all_zero(n, dtype):
     assert np.array_equal(table[:-1], 128 * np.arange(len(table) - 1, dtype=np.uint64))
 
 
-@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("dtype", [np.float32, np.float16, np.uint8])
 @pytest.mark.parametrize("n", [1, 31, 32, 33, 1024, 1030, 4099])
 def test_all_dense(n, dtype):
     s = np.dtype(dtype).itemsize
-    it = np.uint32 if s == 4 else np.uint16
-    x = (np.arange(n, dtype=np.uint64) % 65535 + 1).astype(it).view(dtype)
+    it = {4: np.uint32, 2: np.uint16, 1: np.uint8}[s]
+    x = (np.arange(n, dtype=np.uint64) % (255 if s == 1 else 65535) + 1).astype(it).view(dtype)
     payload, _ = zvc_c.compress(x)
     w = (n + 31) // 32
     assert len(payload) == 4 * w + s * n
@@ -195,13 +205,13 @@ def _check_stream_by_properties(payload, pattern, s):
 
 def sentinel(j, s):
     # non-zero in every byte, distinct per position
-    return (0xA5C30000 | (j + 1)) if s == 4 else (0xA500 | (j + 1))
+    return {4: 0xA5C30000 | (j + 1), 2: 0xA500 | (j + 1), 1: 0xC0 | (j + 1)}[s]
 
 
-@pytest.mark.parametrize("s", [4, 2])
+@pytest.mark.parametrize("s", [4, 2, 1])
 def test_every_pattern_of_tiny_inputs(s):
     # every zero / non-zero pattern of every length up to 16 (4-byte elements; up to 12 for 2-byte ones)
-    it = np.uint32 if s == 4 else np.uint16
+    it = {4: np.uint32, 2: np.uint16, 1: np.uint8}[s]
     for n in range(1, 17 if s == 4 else 13):
         for bits in itertools.product([False, True], repeat=n):
             x = np.array([sentinel(j, s) if b else 0 for j, b in enumerate(bits)], dtype=it)
@@ -211,7 +221,7 @@ def test_every_pattern_of_tiny_inputs(s):
 
 @pytest.mark.parametrize("s", [4, 2])
 def test_all_16bit_patterns_in_both_window_halves(s):
-    it = np.uint32 if s == 4 else np.uint16
+    it = {4: np.uint32, 2: np.uint16, 1: np.uint8}[s]
     pats = np.arange(1 << 16, dtype=np.uint32)
     bits16 = ((pats[:, None] >> np.arange(16)[None, :]) & 1).astype(bool)       # [65536,16]
     lo = np.zeros((1 << 16, 32), dtype=bool)
@@ -233,7 +243,7 @@ def test_all_16bit_patterns_in_both_window_halves(s):
 
 @pytest.mark.parametrize("s", [4, 2])
 def test_walking_one_and_walking_zero(s):
-    it = np.uint32 if s == 4 else np.uint16
+    it = {4: np.uint32, 2: np.uint16, 1: np.uint8}[s]
     for i in range(32):
         one = np.zeros(32, dtype=it)
         one[i] = 0x7B
@@ -264,7 +274,7 @@ def test_every_byte_pattern_in_each_mask_byte():
 # --------------------------------------------------------------------------- #
 # structure: self-delimiting walk, packbits masks, table, layouts
 # --------------------------------------------------------------------------- #
-@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("dtype", [np.float32, np.float16, np.uint8])
 def test_masks_and_values_match_packbits(dtype):
     s = np.dtype(dtype).itemsize
     x = random_sparse(50_000 + 7, 0.37, 5, dtype)
@@ -276,13 +286,13 @@ def test_masks_and_values_match_packbits(dtype):
     assert np.array_equal(vals, zvc_numpy.values(x))
 
 
-@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("dtype", [np.float32, np.float16, np.uint8])
 def test_table_from_independent_chunk_counts(dtype):
     s = np.dtype(dtype).itemsize
     n = 10 * 1024 + 77
     x = random_sparse(n, 0.3, 9, dtype)
     payload, table = zvc_c.compress(x)
-    raw = x.view(np.uint32 if s == 4 else np.uint16)
+    raw = x.view({4: np.uint32, 2: np.uint16, 1: np.uint8}[s])
     k = (n + 1023) // 1024
     assert len(table) == k + 1 == zvc_c.table_entries(n)
     assert table[0] == 0
@@ -362,7 +372,7 @@ def test_too_small_destination_is_reported_and_not_overrun():
     assert payload.tobytes() == full.tobytes()
 
 
-@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("dtype", [np.float32, np.float16, np.uint8])
 @pytest.mark.parametrize("threads", [2, 3, 8])
 def test_threaded_driver_equals_single_thread(dtype, threads):
     for n in (1, 1024, 5 * 1024 + 3, 40_000):
