@@ -19,7 +19,8 @@
  *   concatenation of all records with no header and no padding; its size is
  *   4*ceil(n/32) + s*nnz bytes for n elements of s bytes of which nnz are
  *   non-zero.  A short last window has zero bits for the missing elements.
- *   For 2-byte elements the window is still 32 elements with a 32-bit mask.
+ *   For 2-byte and 1-byte elements the window is still 32 elements with a
+ *   32-bit mask.
  *
  * Framing for parallel decoding (outside the payload): an offset table of
  *   ceil(n/1024)+1 little-endian uint64.  Entry k is the payload offset of
@@ -74,8 +75,9 @@ enum {
     CDMA_ERR_BAD_TICKET = 10
 };
 
-/* element types: only the width matters to the codec (4, 2, 2 bytes) */
-enum { CDMA_F32 = 0, CDMA_F16 = 1, CDMA_BF16 = 2 };
+/* element types: only the width matters to the codec (4, 2, 2, 1 bytes); CDMA_U8
+ * stands for any one-byte element (int8, uint8, an 8-bit float) */
+enum { CDMA_F32 = 0, CDMA_F16 = 1, CDMA_BF16 = 2, CDMA_U8 = 3 };
 
 /* physical layouts of a 4-D activation map (Section II-C); a tag only */
 enum { CDMA_NCHW = 0, CDMA_NHWC = 1, CDMA_CHWN = 2 };
@@ -108,7 +110,7 @@ uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype);
  * prefix-sum / shift / append stages of Section V-B).
  *
  *   d_src           dense tensor, n*s bytes, 16-byte aligned, read only
- *   dtype, layout   CDMA_F32/F16/BF16; CDMA_NCHW/NHWC/CHWN (tag)
+ *   dtype, layout   CDMA_F32/F16/BF16/U8; CDMA_NCHW/NHWC/CHWN (tag)
  *   d_dst           payload out; dst_capacity bytes, 16-byte aligned.  Any
  *                   capacity is accepted; if the payload does not fit the
  *                   call fails with BUFFER_TOO_SMALL having written only
@@ -155,7 +157,8 @@ int cdma_zvc_compress_async(const void* d_src, uint64_t n, int dtype, int layout
  *                (in-place activation) but must not overlap it otherwise, nor
  *                the payload.
  * Everything else, and the payload/table produced, is exactly that of
- * cdma_zvc_compress applied to y.
+ * cdma_zvc_compress applied to y.  CDMA_U8 is refused (UNSUPPORTED_DTYPE): what
+ * "greater than zero" means for a one-byte pattern depends on the type behind it.
  */
 int64_t cdma_zvc_relu_compress(const void* d_src, uint64_t n, int dtype, int layout,
                                void* d_relu_out, void* d_dst, uint64_t dst_capacity,

@@ -27,7 +27,7 @@ from . import zvc_c
 
 def _raw(a: np.ndarray) -> np.ndarray:
     a = np.ascontiguousarray(a).reshape(-1)
-    return a.view(np.uint32 if a.dtype.itemsize == 4 else np.uint16)
+    return a.view({4: np.uint32, 2: np.uint16, 1: np.uint8}[a.dtype.itemsize])
 
 
 def relu_backward(payload: np.ndarray, n: int, dy: np.ndarray) -> np.ndarray:

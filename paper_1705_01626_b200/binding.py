@@ -25,7 +25,7 @@ ERR_CUDA = 8
 ERR_OUT_OF_MEMORY = 9
 ERR_BAD_TICKET = 10
 
-F32, F16, BF16 = 0, 1, 2
+F32, F16, BF16, U8 = 0, 1, 2, 3
 NCHW, NHWC, CHWN = 0, 1, 2
 LAYOUT_CODES = {"NCHW": NCHW, "NHWC": NHWC, "CHWN": CHWN}
 

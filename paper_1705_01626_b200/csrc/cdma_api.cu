@@ -149,6 +149,7 @@ uint32_t cdma_dtype_size(int dtype) {
         case CDMA_F32: return 4;
         case CDMA_F16: return 2;
         case CDMA_BF16: return 2;
+        case CDMA_U8: return 1;
         default: return 0;
     }
 }
@@ -199,6 +200,7 @@ static int compress_enqueue(const void* d_src, uint64_t n, int dtype, int layout
     if (h_result == nullptr) return CDMA_ERR_INVALID_ARG;
     const uint32_t s = cdma_dtype_size(dtype);
     if (overlaps(d_src, n * s, d_dst, dst_capacity)) return CDMA_ERR_INVALID_ARG;
+    if (relu && s == 1) return CDMA_ERR_UNSUPPORTED_DTYPE;
     if (relu && d_relu_out != nullptr) {
         if (!aligned(d_relu_out, 16)) return CDMA_ERR_ALIGNMENT;
         // writing the activation map over its own input is fine; over the payload it is not

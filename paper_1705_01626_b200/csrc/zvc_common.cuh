@@ -127,17 +127,19 @@ __device__ inline void report_decode_error(uint64_t* ws, const LaunchCtl& ctl, u
     __threadfence_system();
 }
 
-// Launchers (defined next to their kernels).  elem_size is 2 or 4.  src_on_device
+// Launchers (defined next to their kernels).  elem_size is 1, 2 or 4.  src_on_device
 // is false when the input lies in mapped host memory: the kernels then leave out
 // their L2 prefetches, which would fetch every line over the host link twice,
 // and compression takes the kernel that loads with plain instructions.
 cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst,
                                 uint64_t cap, uint64_t* d_table, uint64_t* d_ws, const LaunchCtl& ctl,
                                 cudaStream_t stream, bool src_on_device = true);
-// The kernel for device-resident 2-byte tensors of at least one tile (zvc_compress_rows.cu).
-bool zvc_compress_rows_usable(const void* d_src, uint64_t n, uint32_t elem_size);
-cudaError_t launch_zvc_compress_rows(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
-                                     uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream);
+// The row-per-thread kernel for 2-byte and 1-byte elements (zvc_compress_rows.cu).  With use_tma (device
+// memory, at least one tile) the tile comes in by one TMA tensor copy; without, by plain loads.
+bool zvc_compress_rows_tma_usable(const void* d_src, uint64_t n, uint32_t elem_size);
+cudaError_t launch_zvc_compress_rows(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst, uint64_t cap,
+                                     uint64_t* d_table, uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream,
+                                     bool use_tma);
 void preload_compress_rows_kernel();
 void preload_compress_kernels();     // load every compression kernel now rather than at its first launch
 cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t elem_size, uint32_t nan_above,
@@ -147,6 +149,8 @@ cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t ele
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
                                   const LaunchCtl& ctl, cudaStream_t stream, bool src_on_device = true);
+cudaError_t launch_zvc_decompress_u8(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                     void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream);
 cudaError_t launch_zvc_relu_backward(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
                                      uint32_t elem_size, const void* d_dy, void* d_dx, uint64_t* d_ws,
                                      const LaunchCtl& ctl, cudaStream_t stream);

@@ -500,9 +500,11 @@ cudaError_t launch_zvc_compress(const void* d_src, uint64_t n, uint32_t elem_siz
                                 uint64_t cap, uint64_t* d_table, uint64_t* d_ws, const LaunchCtl& ctl,
                                 cudaStream_t stream, bool src_on_device) {
     if (num_tiles_of(n) == 0) return cudaSuccess;
-    // 2-byte elements in device memory, at least one tile: the row-per-thread kernel with TMA loads
-    if (src_on_device && zvc_compress_rows_usable(d_src, n, elem_size))
-        return launch_zvc_compress_rows(d_src, n, d_dst, cap, d_table, d_ws, ctl, stream);
+    // 2-byte and 1-byte elements in device memory, at least one tile: the row-per-thread kernel with TMA loads;
+    // 1-byte elements have no other kernel and take it without the tensor copy otherwise
+    const bool tma = src_on_device && zvc_compress_rows_tma_usable(d_src, n, elem_size);
+    if (tma || elem_size == 1)
+        return launch_zvc_compress_rows(d_src, n, elem_size, d_dst, cap, d_table, d_ws, ctl, stream, tma);
     const cudaError_t e =
         (elem_size == 4)
             ? launch_typed<uint32_t, kTileChunks>(zvc_compress_kernel<uint32_t, false>, d_src, n, d_dst, cap,

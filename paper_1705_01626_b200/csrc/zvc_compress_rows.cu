@@ -1,16 +1,17 @@
-// Zero-value compression (Section V-A) of 2-byte elements that live in device
-// memory: one thread owns one row of 128 bytes of the input -- two windows of 32
-// elements -- so that the whole record of a window (compare, count, shift, append:
-// the stages of Section V-B, Fig. 10a) is built by one thread from its own
-// registers, with no work repeated across lanes and no cross-lane traffic.  With
-// half the bytes per element, the per-element cost is what bounds this width;
-// 4-byte elements stay with the kernel in zvc_compress.cu, which is faster there.
+// Zero-value compression (Section V-A) of 2-byte and 1-byte elements that live in
+// device memory: one thread owns one row of 128 bytes of the input -- two windows
+// of 32 two-byte elements, or four of 32 one-byte elements -- so that the whole
+// record of a window (compare, count, shift, append: the stages of Section V-B,
+// Fig. 10a) is built by one thread from its own registers, with no work repeated
+// across lanes and no cross-lane traffic.  With fewer bytes per element, the
+// per-element cost is what bounds these widths; 4-byte elements stay with the
+// kernel in zvc_compress.cu, which is faster there.
 //
-// A CTA compresses a tile of 256 rows (32 KB, 16 chunks).  Order of work:
+// A CTA compresses a tile of 256 rows (32 KB: 16 or 32 chunks).  Order of work:
 //   1. load: one TMA tensor copy brings the tile into shared memory (128-byte
 //      swizzle, so that thread t's reads of row t do not collide with its
 //      neighbours'); each thread then takes its row into 32 registers;
-//   2. count: two masks and the number of non-zero elements per thread; a scan
+//   2. count: the row's masks and number of non-zero elements per thread; a scan
 //      over the CTA gives every record its place in the tile, and the tile's
 //      size is published at once for the tiles behind it (single-pass decoupled
 //      look-back);
@@ -20,6 +21,8 @@
 //   5. copy: the CTA moves the staged bytes to the payload with aligned 16-byte
 //      stores, realigning in registers.
 #include <cuda.h>
+
+#include <cstring>
 
 #include "zvc_common.cuh"
 #include "lookback.cuh"
@@ -31,8 +34,8 @@ namespace {
 
 constexpr uint32_t kRows = kTileThreads;               // rows of 128 bytes per tile, one per thread
 constexpr uint32_t kRowBytes = 128;
-constexpr uint32_t kRowElems = kRowBytes / 2;
-constexpr uint32_t kStageBytes = kRows * 136 + 32;     // largest tile output (every element non-zero) + slack
+// largest tile output (every element non-zero: a mask per window and the row itself) + slack
+constexpr uint32_t stage_bytes(uint32_t elem_size) { return kRows * (kRowBytes + 4 * (4 / elem_size)) + 32; }
 // Tiles follow the block index and blocks are dispatched in that order, so the tile this many places
 // further on will be picked up by a CTA that starts about half a CTA lifetime from now.
 constexpr uint32_t kPrefetchAheadTiles = 370;
@@ -78,6 +81,35 @@ __device__ __forceinline__ void sts_mask(uint32_t q, uint32_t m) {
                  ::"r"(q), "r"(m) : "memory");
 }
 
+// ---- 1-byte elements ---------------------------------------------------------------------------
+// the 4 "byte is non-zero" bits of a word (byte 0 = bit 0)
+__device__ __forceinline__ uint32_t nonzero_bytes(uint32_t w) {
+    const uint32_t t = (((w & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w) & 0x80808080u;   // 0x80 in every non-zero byte
+    return (((t >> 7) * 0x00204081u) >> 21) & 15u;                               // bits 0, 8, 16, 24 -> 0, 1, 2, 3
+}
+// mask of a window of 32 one-byte elements held in 8 words
+__device__ __forceinline__ uint32_t mask_of_bytes(const uint32_t* w) {
+    uint32_t m = 0;
+#pragma unroll
+    for (uint32_t j = 0; j < 8; ++j) m |= nonzero_bytes(w[j]) << (4 * j);
+    return m;
+}
+// append the non-zero bytes of w (lowest first) at q + 4
+__device__ __forceinline__ void append_bytes(uint32_t& q, uint32_t w) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 h;\n\t"
+                 "prmt.b32 h, %1, 0, 0x4440;\n\tsetp.ne.u32 p, h, 0;\n\t@p st.shared.u8 [%0+4], h;\n\t@p add.u32 %0, %0, 1;\n\t"
+                 "prmt.b32 h, %1, 0, 0x4441;\n\tsetp.ne.u32 p, h, 0;\n\t@p st.shared.u8 [%0+4], h;\n\t@p add.u32 %0, %0, 1;\n\t"
+                 "prmt.b32 h, %1, 0, 0x4442;\n\tsetp.ne.u32 p, h, 0;\n\t@p st.shared.u8 [%0+4], h;\n\t@p add.u32 %0, %0, 1;\n\t"
+                 "prmt.b32 h, %1, 0, 0x4443;\n\tsetp.ne.u32 p, h, 0;\n\t@p st.shared.u8 [%0+4], h;\n\t@p add.u32 %0, %0, 1;\n\t}"
+                 : "+r"(q) : "r"(w) : "memory");
+}
+// a mask word at any shared byte address
+__device__ __forceinline__ void sts_mask_bytes(uint32_t q, uint32_t m) {
+    asm volatile("{\n\t.reg .b32 h;\n\tst.shared.u8 [%0], %1;\n\tshr.u32 h, %1, 8;\n\tst.shared.u8 [%0+1], h;\n\t"
+                 "shr.u32 h, %1, 16;\n\tst.shared.u8 [%0+2], h;\n\tshr.u32 h, %1, 24;\n\tst.shared.u8 [%0+3], h;\n\t}"
+                 ::"r"(q), "r"(m) : "memory");
+}
+
 // Bounded wait for the tile to land.  Returns false when the limit ran out.
 __device__ __forceinline__ bool wait_tile(uint32_t mbar, uint64_t limit_ns) {
     uint32_t done = 0;
@@ -99,11 +131,15 @@ __device__ __forceinline__ bool wait_tile(uint32_t mbar, uint64_t limit_ns) {
 // that order, so a tile only ever waits for blocks that were dispatched before it (the
 // assumption single-pass scans rest on); should it ever not hold, the bounded wait in the
 // walk turns it into CDMA_ERR_TIMEOUT.
+// S = element size (2 or 1).
+template <uint32_t S>
 __global__ void __launch_bounds__(kTileThreads, kMinCtasPerSm)
-zvc_compress_rows_kernel_u16(const __grid_constant__ CUtensorMap tmap, const uint16_t* __restrict__ src, uint64_t n,
-                             uint8_t* __restrict__ dst, uint64_t cap, uint64_t* __restrict__ table,
-                             uint64_t* __restrict__ ws, const LaunchCtl ctl, uint32_t num_tiles, uint64_t num_chunks,
-                             uint64_t full_rows) {
+zvc_compress_rows_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t* __restrict__ src, uint64_t n,
+                         uint8_t* __restrict__ dst, uint64_t cap, uint64_t* __restrict__ table,
+                         uint64_t* __restrict__ ws, const LaunchCtl ctl, uint32_t num_tiles, uint64_t num_chunks,
+                         uint64_t full_rows, uint32_t use_tma) {
+    constexpr uint32_t WPR = 4 / S;                              // windows per row: 2 or 4
+    constexpr uint32_t WW = 8 * S;                               // words per window: 16 or 8
     extern __shared__ __align__(1024) uint8_t smem_raw[];          // input tile, then the staged output
     __shared__ __align__(8) uint64_t s_mbar;
     __shared__ uint32_t s_warp_bytes[kTileThreads / 32];
@@ -121,33 +157,37 @@ zvc_compress_rows_kernel_u16(const __grid_constant__ CUtensorMap tmap, const uin
     const uint64_t row0 = static_cast<uint64_t>(tile) * kRows;
 
     // ---- 1. load -------------------------------------------------------------------------------
+    // (use_tma is 0 for tensors the tensor copy cannot serve -- less than one row, or in host memory:
+    // every thread then fetches its row with plain loads further down)
     if (tid == 0) {
         s_late = 0;
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar) : "memory");
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (use_tma) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar) : "memory");
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
     }
     __syncthreads();
-    if (tid == 0) {
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(kTileBytes) : "memory");
-        // rows past the end of the tensor map (the last tile only) arrive as zeros
-        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                     ::"r"(s_stage), "l"(&tmap), "r"(0), "r"(static_cast<int32_t>(row0)), "r"(mbar) : "memory");
-    } else if (tid == 32) {
-        // asking L2 for a later tile now turns that tile's load into L2 hits; every line still comes
-        // from DRAM exactly once
-        const uint64_t prow = row0 + static_cast<uint64_t>(kPrefetchAheadTiles) * kRows;
-        if (prow + kRows <= full_rows)
-            asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-                         ::"l"(&tmap), "r"(0), "r"(static_cast<int32_t>(prow)) : "memory");
-    }
-    // (a thread whose wait ran out goes on with whatever shared memory holds; the CTA decides
-    // together behind the next barrier)
-    if (!wait_tile(mbar, ctl.wait_limit_ns)) s_late = 1;
-
-    // thread t takes row t: eight 16-byte pieces, piece i stored at position i ^ (t & 7) by the swizzle
     uint32_t e[32];
-    {
+    if (use_tma) {
+        if (tid == 0) {
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(kTileBytes) : "memory");
+            // rows past the end of the tensor map (the last tile only) arrive as zeros
+            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                         ::"r"(s_stage), "l"(&tmap), "r"(0), "r"(static_cast<int32_t>(row0)), "r"(mbar) : "memory");
+        } else if (tid == 32) {
+            // asking L2 for a later tile now turns that tile's load into L2 hits; every line still comes
+            // from DRAM exactly once
+            const uint64_t prow = row0 + static_cast<uint64_t>(kPrefetchAheadTiles) * kRows;
+            if (prow + kRows <= full_rows)
+                asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                             ::"l"(&tmap), "r"(0), "r"(static_cast<int32_t>(prow)) : "memory");
+        }
+        // (a thread whose wait ran out goes on with whatever shared memory holds; the CTA decides
+        // together behind the next barrier)
+        if (!wait_tile(mbar, ctl.wait_limit_ns)) s_late = 1;
+
+        // thread t takes row t: eight 16-byte pieces, piece i stored at position i ^ (t & 7) by the swizzle
         const uint32_t row_addr = s_stage + kRowBytes * tid;
         const uint32_t sw = tid & 7u;
 #pragma unroll
@@ -155,28 +195,44 @@ zvc_compress_rows_kernel_u16(const __grid_constant__ CUtensorMap tmap, const uin
             const uint4 v = lds128(row_addr + 16u * (i ^ sw));
             e[4 * i + 0] = v.x; e[4 * i + 1] = v.y; e[4 * i + 2] = v.z; e[4 * i + 3] = v.w;
         }
+    } else {
+#pragma unroll
+        for (uint32_t i = 0; i < 32; ++i) e[i] = 0;
+        if (row0 + tid < full_rows) {
+            const uint4* rp = reinterpret_cast<const uint4*>(src + (row0 + tid) * kRowBytes);
+#pragma unroll
+            for (uint32_t i = 0; i < 8; ++i) {
+                const uint4 v = __ldcs(rp + i);
+                e[4 * i + 0] = v.x; e[4 * i + 1] = v.y; e[4 * i + 2] = v.z; e[4 * i + 3] = v.w;
+            }
+        }
     }
     const uint64_t row = row0 + tid;
     // windows of this row that exist (the tensor may end inside the last tile)
     const uint64_t total_windows = (n + kWindow - 1) / kWindow;
-    const uint64_t w_first = 2 * row;
-    const uint32_t nwin = w_first >= total_windows ? 0u : (total_windows - w_first >= 2 ? 2u : 1u);
+    const uint64_t w_first = WPR * row;
+    const uint32_t nwin = w_first >= total_windows ? 0u
+                          : (total_windows - w_first >= WPR ? WPR : static_cast<uint32_t>(total_windows - w_first));
     if (row >= full_rows && nwin != 0) {
-        // the one row that is only partly inside the tensor: plain guarded loads
-        const uint64_t e0 = row * kRowElems;
+        // the one row that is only partly inside the tensor: plain guarded loads, byte by byte
+        const uint64_t b0 = row * kRowBytes, nbytes = n * S;
 #pragma unroll
         for (uint32_t i = 0; i < 32; ++i) {
-            const uint64_t j = e0 + 2 * i;
-            const uint32_t lo = j < n ? src[j] : 0u;
-            const uint32_t hi = j + 1 < n ? src[j + 1] : 0u;
-            e[i] = lo | (hi << 16);
+            uint32_t v = 0;
+            for (uint32_t b = 0; b < 4; ++b)
+                if (b0 + 4 * i + b < nbytes) v |= static_cast<uint32_t>(src[b0 + 4 * i + b]) << (8 * b);
+            e[i] = v;
         }
     }
 
     // ---- 2. count ------------------------------------------------------------------------------
-    const uint32_t mask_a = interleave16(flags_of(e));
-    const uint32_t mask_b = interleave16(flags_of(e + 16));
-    const uint32_t rec_bytes = (nwin > 0 ? 4u + 2u * __popc(mask_a) : 0u) + (nwin > 1 ? 4u + 2u * __popc(mask_b) : 0u);
+    uint32_t mask[WPR];
+    uint32_t rec_bytes = 0;
+#pragma unroll
+    for (uint32_t k = 0; k < WPR; ++k) {
+        mask[k] = (S == 2) ? interleave16(flags_of(e + WW * k)) : mask_of_bytes(e + WW * k);
+        if (k < nwin) rec_bytes += 4u + S * __popc(mask[k]);
+    }
     // place of every thread's records in the tile: scan over the warp, then over the warps
     uint32_t incl = rec_bytes;
 #pragma unroll
@@ -190,7 +246,7 @@ zvc_compress_rows_kernel_u16(const __grid_constant__ CUtensorMap tmap, const uin
         // The copy is late beyond the limit.  One more bounded wait, so that it cannot write into shared
         // memory this CTA has already handed back; then the launch fails the way a look-back time-out
         // does: the tile marks itself, so that the tiles behind it stop as well.
-        (void)wait_tile(mbar, ctl.wait_limit_ns);
+        if (use_tma) (void)wait_tile(mbar, ctl.wait_limit_ns);
         if (tid == 0) {
             publish_prefix(ws, ctl, tile, true, 0);
             if (tile == num_tiles - 1) publish_result(ws, ctl, 0, CDMA_ERR_TIMEOUT);
@@ -209,16 +265,18 @@ zvc_compress_rows_kernel_u16(const __grid_constant__ CUtensorMap tmap, const uin
 
     // ---- 3. assemble -----------------------------------------------------------------------------
     uint32_t q = s_stage + rec_off;
-    if (nwin > 0) {
-        sts_mask(q, mask_a);
 #pragma unroll
-        for (uint32_t i = 0; i < 16; ++i) append_pair(q, e[i]);
-        q += 4;
-    }
-    if (nwin > 1) {
-        sts_mask(q, mask_b);
+    for (uint32_t k = 0; k < WPR; ++k) {
+        if (k < nwin) {
+            if (S == 2) sts_mask(q, mask[k]);
+            else sts_mask_bytes(q, mask[k]);
 #pragma unroll
-        for (uint32_t i = 16; i < 32; ++i) append_pair(q, e[i]);
+            for (uint32_t i = 0; i < WW; ++i) {
+                if (S == 2) append_pair(q, e[WW * k + i]);
+                else append_bytes(q, e[WW * k + i]);
+            }
+            q += 4;
+        }
     }
 
     // ---- 4. the tile's place in the stream -------------------------------------------------------
@@ -228,12 +286,13 @@ zvc_compress_rows_kernel_u16(const __grid_constant__ CUtensorMap tmap, const uin
     if (s_failed) return;
     const uint64_t base = s_base;
 
-    // offset-table entries: a chunk is 32 windows = 16 rows
-    const uint64_t chunk = static_cast<uint64_t>(tile) * (kRows / 16) + 2 * warp + (lane >> 4);
-    if ((lane & 15u) == 0 && chunk < num_chunks) table[chunk] = base + rec_off;
+    // offset-table entries: a chunk is 32 windows = 32 / WPR rows
+    constexpr uint32_t kChunkRows = 32 / WPR;
+    const uint64_t chunk = static_cast<uint64_t>(tile) * (kRows / kChunkRows) + WPR * warp + lane / kChunkRows;
+    if (lane % kChunkRows == 0 && chunk < num_chunks) table[chunk] = base + rec_off;
 
     // ---- 5. copy the staged bytes to their place, below the capacity ------------------------------
-    copy_out<2, kTileThreads>(s_stage, smem_raw, dst, base, s_room);
+    copy_out<S, kTileThreads>(s_stage, smem_raw, dst, base, s_room);
 }
 
 // The driver's tensor-map encoder, looked up once (no link-time dependency on the driver library).
@@ -258,39 +317,46 @@ EncodeTiledFn encode_tiled() {
 
 void preload_compress_rows_kernel() {
     cudaFuncAttributes a;
-    (void)cudaFuncGetAttributes(&a, zvc_compress_rows_kernel_u16);
+    (void)cudaFuncGetAttributes(&a, zvc_compress_rows_kernel<2>);
+    (void)cudaFuncGetAttributes(&a, zvc_compress_rows_kernel<1>);
     (void)encode_tiled();
 }
 
-bool zvc_compress_rows_usable(const void* d_src, uint64_t n, uint32_t elem_size) {
-    // 2-byte elements, at least one whole tile, rows addressable with 32-bit coordinates, and an
+bool zvc_compress_rows_tma_usable(const void* d_src, uint64_t n, uint32_t elem_size) {
+    // 2-byte or 1-byte elements, at least one whole tile, rows addressable with 32-bit coordinates, and an
     // encoder to describe them
     const uint64_t full_rows = n * elem_size / kRowBytes;
-    return elem_size == 2 && full_rows >= kRows && full_rows < (1ull << 31) &&
+    return (elem_size == 2 || elem_size == 1) && full_rows >= kRows && full_rows < (1ull << 31) &&
            (reinterpret_cast<uintptr_t>(d_src) & 15) == 0 && encode_tiled() != nullptr;
 }
 
-cudaError_t launch_zvc_compress_rows(const void* d_src, uint64_t n, void* d_dst, uint64_t cap, uint64_t* d_table,
-                                     uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream) {
-    const uint64_t bytes = n * 2;
+cudaError_t launch_zvc_compress_rows(const void* d_src, uint64_t n, uint32_t elem_size, void* d_dst, uint64_t cap,
+                                     uint64_t* d_table, uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream,
+                                     bool use_tma) {
+    const uint64_t bytes = n * elem_size;
     const uint64_t full_rows = bytes / kRowBytes;
     const uint64_t tiles = (bytes + kTileBytes - 1) / kTileBytes;
-    // the tensor as rows of 32 words; a box is one tile; 128-byte swizzle
     CUtensorMap tmap;
-    const cuuint64_t dims[2] = {kRowBytes / 4, full_rows};
-    const cuuint64_t strides[1] = {kRowBytes};
-    const cuuint32_t box[2] = {kRowBytes / 4, kRows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = encode_tiled()(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(d_src), dims, strides,
-                                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    const cudaError_t oe = opt_in_shared_memory(reinterpret_cast<const void*>(zvc_compress_rows_kernel_u16), kStageBytes);
+    memset(&tmap, 0, sizeof(tmap));
+    if (use_tma) {
+        // the tensor as rows of 32 words; a box is one tile; 128-byte swizzle
+        const cuuint64_t dims[2] = {kRowBytes / 4, full_rows};
+        const cuuint64_t strides[1] = {kRowBytes};
+        const cuuint32_t box[2] = {kRowBytes / 4, kRows};
+        const cuuint32_t estr[2] = {1, 1};
+        const CUresult r = encode_tiled()(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(d_src), dims,
+                                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
+    auto kernel = elem_size == 2 ? zvc_compress_rows_kernel<2> : zvc_compress_rows_kernel<1>;
+    const uint32_t smem = stage_bytes(elem_size);
+    const cudaError_t oe = opt_in_shared_memory(reinterpret_cast<const void*>(kernel), smem);
     if (oe != cudaSuccess) return oe;
     timing_before_launch(stream);
-    zvc_compress_rows_kernel_u16<<<static_cast<unsigned>(tiles), kTileThreads, kStageBytes, stream>>>(
-        tmap, static_cast<const uint16_t*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws, ctl,
-        static_cast<uint32_t>(tiles), num_chunks_of(n), full_rows);
+    kernel<<<static_cast<unsigned>(tiles), kTileThreads, smem, stream>>>(
+        tmap, static_cast<const uint8_t*>(d_src), n, static_cast<uint8_t*>(d_dst), cap, d_table, d_ws, ctl,
+        static_cast<uint32_t>(tiles), num_chunks_of(n), full_rows, use_tma ? 1u : 0u);
     timing_after_launch(stream);
     count_kernel_launch();
     return cudaGetLastError();

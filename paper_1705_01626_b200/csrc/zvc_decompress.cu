@@ -433,6 +433,12 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
     if (chunks == 0) return cudaSuccess;
     const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
     timing_before_launch(stream);
+    if (elem_size == 1) {
+        const cudaError_t e = launch_zvc_decompress_u8(d_src, src_bytes, d_table, n, d_dst, d_ws, ctl, stream);
+        timing_after_launch(stream);
+        count_kernel_launch();
+        return e;
+    }
     if (elem_size == 4) {
         // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
         const bool prefetch = src_on_device && src_bytes >= (n * 4) / 5;

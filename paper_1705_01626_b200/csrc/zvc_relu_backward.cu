@@ -26,11 +26,16 @@ namespace {
 constexpr uint32_t kBwdWarps = 8;
 
 __device__ __forceinline__ uint32_t ld_mask(const uint8_t* p, uint32_t elem_size) {
-    // a mask starts on an element boundary: 4-byte aligned for 4-byte elements, 2-byte aligned otherwise
+    // a mask starts on an element boundary: 4-byte aligned for 4-byte elements, 2-byte aligned for 2-byte
+    // ones, anywhere for 1-byte ones
     if (elem_size == 4) return __ldg(reinterpret_cast<const uint32_t*>(p));
-    const uint32_t lo = __ldg(reinterpret_cast<const uint16_t*>(p));
-    const uint32_t hi = __ldg(reinterpret_cast<const uint16_t*>(p + 2));
-    return lo | (hi << 16);
+    if (elem_size == 2) {
+        const uint32_t lo = __ldg(reinterpret_cast<const uint16_t*>(p));
+        const uint32_t hi = __ldg(reinterpret_cast<const uint16_t*>(p + 2));
+        return lo | (hi << 16);
+    }
+    return static_cast<uint32_t>(__ldg(p)) | (static_cast<uint32_t>(__ldg(p + 1)) << 8) |
+           (static_cast<uint32_t>(__ldg(p + 2)) << 16) | (static_cast<uint32_t>(__ldg(p + 3)) << 24);
 }
 
 template <uint32_t S>
@@ -71,10 +76,10 @@ zvc_relu_backward_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, co
             // any word of the line that lies inside the payload
             const uint64_t at = a < lo ? lo : a;
             uint32_t v;
-            asm volatile("ld.global.ca.u16 %0, [%1];" : "=r"(v) : "l"(src + at) : "memory");
+            asm volatile("ld.global.ca.u8 %0, [%1];" : "=r"(v) : "l"(src + at) : "memory");
             sink ^= v;
         }
-        if (sink == 0x9e3779b9u) asm volatile("" ::: "memory");     // keeps the loads; never true for 16-bit values
+        if (sink == 0x9e3779b9u) asm volatile("" ::: "memory");     // keeps the loads; never true for 8-bit values
     }
 
     // ---- the walk: lane w ends up with the mask of window w ----------------------------------------
@@ -114,12 +119,18 @@ zvc_relu_backward_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, co
                 v.y = (bits & 2u) ? v.y : 0u;
                 v.z = (bits & 4u) ? v.z : 0u;
                 v.w = (bits & 8u) ? v.w : 0u;
-            } else {
+            } else if (S == 2) {
                 // two elements per word: keep masks from two bits each
                 v.x &= ((bits & 1u) ? 0xffffu : 0u) | ((bits & 2u) ? 0xffff0000u : 0u);
                 v.y &= ((bits & 4u) ? 0xffffu : 0u) | ((bits & 8u) ? 0xffff0000u : 0u);
                 v.z &= ((bits & 16u) ? 0xffffu : 0u) | ((bits & 32u) ? 0xffff0000u : 0u);
                 v.w &= ((bits & 64u) ? 0xffffu : 0u) | ((bits & 128u) ? 0xffff0000u : 0u);
+            } else {
+                // four elements per word: 4 bits -> 4 byte masks (bit k to bit 8k, then times 255)
+                v.x &= (((bits >> 0) & 15u) * 0x00204081u & 0x01010101u) * 255u;
+                v.y &= (((bits >> 4) & 15u) * 0x00204081u & 0x01010101u) * 255u;
+                v.z &= (((bits >> 8) & 15u) * 0x00204081u & 0x01010101u) * 255u;
+                v.w &= (((bits >> 12) & 15u) * 0x00204081u & 0x01010101u) * 255u;
             }
             __stcs(out + 32 * r, v);
         }
@@ -131,7 +142,8 @@ zvc_relu_backward_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes, co
             if (j < n) {
                 const bool keep = (m >> lane) & 1u;
                 if (S == 4) reinterpret_cast<uint32_t*>(dx)[j] = keep ? reinterpret_cast<const uint32_t*>(dy)[j] : 0u;
-                else reinterpret_cast<uint16_t*>(dx)[j] = keep ? reinterpret_cast<const uint16_t*>(dy)[j] : uint16_t(0);
+                else if (S == 2) reinterpret_cast<uint16_t*>(dx)[j] = keep ? reinterpret_cast<const uint16_t*>(dy)[j] : uint16_t(0);
+                else dx[j] = keep ? dy[j] : uint8_t(0);
             }
         }
     }
@@ -150,8 +162,12 @@ cudaError_t launch_zvc_relu_backward(const void* d_src, uint64_t src_bytes, cons
         zvc_relu_backward_kernel<4><<<grid, 32 * kBwdWarps, 0, stream>>>(
             static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<const uint8_t*>(d_dy),
             static_cast<uint8_t*>(d_dx), d_ws, ctl, chunks);
-    else
+    else if (elem_size == 2)
         zvc_relu_backward_kernel<2><<<grid, 32 * kBwdWarps, 0, stream>>>(
+            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<const uint8_t*>(d_dy),
+            static_cast<uint8_t*>(d_dx), d_ws, ctl, chunks);
+    else
+        zvc_relu_backward_kernel<1><<<grid, 32 * kBwdWarps, 0, stream>>>(
             static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<const uint8_t*>(d_dy),
             static_cast<uint8_t*>(d_dx), d_ws, ctl, chunks);
     timing_after_launch(stream);

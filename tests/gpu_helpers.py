@@ -6,16 +6,16 @@ import torch
 
 from paper_1705_01626_b200 import binding as B
 
-DT = {torch.float32: B.F32, torch.float16: B.F16, torch.bfloat16: B.BF16}
-NP_RAW = {4: np.uint32, 2: np.uint16}
+DT = {torch.float32: B.F32, torch.float16: B.F16, torch.bfloat16: B.BF16, torch.uint8: B.U8}
+NP_RAW = {4: np.uint32, 2: np.uint16, 1: np.uint8}
+TORCH_RAW = {4: torch.int32, 2: torch.int16, 1: torch.uint8}
 CANARY = 0xA7
 
 
 def raw_numpy(x: torch.Tensor) -> np.ndarray:
     """Host copy of a tensor's bit patterns as a flat unsigned array."""
     flat = x.detach().contiguous().view(-1)
-    it = torch.int32 if x.element_size() == 4 else torch.int16
-    return flat.view(it).cpu().numpy().view(NP_RAW[x.element_size()])
+    return flat.view(TORCH_RAW[x.element_size()]).cpu().numpy().view(NP_RAW[x.element_size()])
 
 
 class DeviceCodec:

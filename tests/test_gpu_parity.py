@@ -23,11 +23,11 @@ SIZES = [0, 1, 31, 32, 33, 63, 64, 65, 1023, 1024, 1025, 2047, 2048, 2049,
 
 
 def make(n, density, seed, dtype):
-    it = np.uint32 if dtype == torch.float32 else np.uint16
+    it = {torch.float32: np.uint32, torch.float16: np.uint16, torch.uint8: np.uint8}[dtype]
     rng = np.random.default_rng(seed)
     raw = rng.integers(1, np.iinfo(it).max, size=n, dtype=it, endpoint=True)
     raw[rng.random(n) >= density] = 0
-    t = torch.from_numpy(raw.view(np.int32 if it == np.uint32 else np.int16)).cuda()
+    t = torch.from_numpy(raw.view({np.uint32: np.int32, np.uint16: np.int16, np.uint8: np.uint8}[it])).cuda()
     return t.view(dtype), raw
 
 
@@ -41,29 +41,29 @@ def check_against_oracle(x: torch.Tensor, raw: np.ndarray):
     assert codec.payload_numpy(c).tobytes() == want_payload.tobytes()
     assert np.array_equal(codec.table_numpy(), want_table)
     assert codec.canaries_intact()
-    out = torch.full_like(x.view(-1), 1.25 if x.dtype != torch.float32 else 3.5)
+    out = torch.full_like(x.view(-1), 77 if x.dtype == torch.uint8 else (1.25 if x.dtype != torch.float32 else 3.5))
     r = codec.decompress(out, c)
     assert r == n * x.element_size(), B.status_string(r)
     assert raw_numpy(out).tobytes() == raw.tobytes()
     # and the GPU decoder accepts the oracle's own stream
     codec.load(want_payload, want_table)
-    out.fill_(7.0)
+    out.fill_(7)
     assert codec.decompress(out, len(want_payload)) == n * x.element_size()
     assert raw_numpy(out).tobytes() == raw.tobytes()
     return c
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
-@pytest.mark.parametrize("n", SIZES)
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.uint8])
+@pytest.mark.parametrize("n", SIZES + [4 * TILE - 1, 4 * TILE + 1, 9 * TILE + 77])
 def test_sizes_and_tails(n, dtype):
     for seed, density in enumerate([0.1, 0.5, 0.93]):
         x, raw = make(n, density, 1000 * seed + n, dtype)
         check_against_oracle(x, raw)
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16, torch.uint8])
 def test_all_zero_and_all_dense(dtype):
-    n = 3 * TILE + 100
+    n = 3 * TILE + 100 if dtype != torch.uint8 else 9 * TILE + 100
     z = torch.zeros(n, dtype=dtype, device="cuda")
     c = check_against_oracle(z, raw_numpy(z))
     assert c == 4 * ((n + 31) // 32)
@@ -84,9 +84,9 @@ def test_every_16bit_mask_pattern_in_both_halves():
     lo = np.zeros((1 << 16, 32), dtype=bool); lo[:, :16] = bits16
     hi = np.zeros((1 << 16, 32), dtype=bool); hi[:, 16:] = bits16
     pattern = np.concatenate([lo, hi]).reshape(-1)
-    for it, dt in ((np.uint32, torch.float32), (np.uint16, torch.float16)):
+    for it, dt in ((np.uint32, torch.float32), (np.uint16, torch.float16), (np.uint8, torch.uint8)):
         raw = np.where(pattern, (np.arange(pattern.size) % 251 + 1), 0).astype(it)
-        x = torch.from_numpy(raw.view(np.int32 if it == np.uint32 else np.int16)).cuda().view(dt)
+        x = torch.from_numpy(raw.view({np.uint32: np.int32, np.uint16: np.int16, np.uint8: np.uint8}[it])).cuda().view(dt)
         check_against_oracle(x, raw)
 
 
@@ -126,12 +126,12 @@ def test_capacity_too_small_is_reported_without_overrun():
     assert codec.compress(x) == len(want)
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.uint8])
 def test_capacity_at_tile_and_line_boundaries(dtype):
     """Capacities that end on, just before and just after the places where the copy-out
     changes row or tile: everything below the capacity is the stream's prefix, nothing
     above it is touched."""
-    x, raw = make(5 * TILE + 3 * 1024 + 41, 0.45, 17, dtype)
+    x, raw = make((5 * TILE + 3 * 1024) * (4 if dtype == torch.uint8 else 1) + 41, 0.45, 17, dtype)
     want, table = zvc_c.compress(raw)
     s = x.element_size()
     tile_starts = [int(table[k]) for k in range(0, len(table) - 1, 8)]      # first chunk of every 8th
@@ -150,7 +150,7 @@ def test_capacity_at_tile_and_line_boundaries(dtype):
         assert (codec.payload_numpy(cap)[whole:] == CANARY).all(), cap
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.uint8])
 def test_corrupt_table_and_stream_are_rejected_without_faulting(dtype):
     x, raw = make(4 * TILE + 300, 0.4, 11, dtype)
     n = x.numel()
@@ -194,7 +194,7 @@ def test_corrupt_table_and_stream_are_rejected_without_faulting(dtype):
     assert codec.decompress(torch.zeros(40, device="cuda"), len(bad)) == -B.ERR_CORRUPT_STREAM
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.uint8])
 def test_garbage_streams_never_fault(dtype):
     """Streams that are not streams: random bytes, all-ones masks (records as long as they get),
     zeros, behind tables whose chunk sizes are possible.  The answer is CORRUPT_STREAM (or, by
@@ -225,11 +225,11 @@ def test_garbage_streams_never_fault(dtype):
             payload = rng.integers(0, 2, size=total, dtype=np.uint8) * 0xFF
         codec = DeviceCodec(n, dtype)
         codec.load(payload, table)
-        out = torch.full((n + guard,), 7.0, dtype=dtype, device="cuda")
+        out = torch.full((n + guard,), 7, dtype=dtype, device="cuda")
         r = codec.decompress(out, total)
         assert r in (-B.ERR_CORRUPT_STREAM, n * s), B.status_string(r)
         assert codec.canaries_intact()
-        assert bool((out[n:] == 7.0).all())
+        assert bool((out[n:] == 7).all())
     # the library still works afterwards
     x, raw = make(n, 0.3, 2, dtype)
     check_against_oracle(x, raw)

@@ -38,6 +38,15 @@ def test_matches_the_oracle(dtype, n):
         run(x, dy)
 
 
+def test_one_byte_elements():
+    for n, density in [(5, 1.0), (1024, 0.5), (70_000 + 3, 0.2)]:
+        raw = np.random.default_rng(n).integers(1, 255, size=n, dtype=np.uint8)
+        raw[np.random.default_rng(n + 1).random(n) >= density] = 0
+        x = torch.from_numpy(raw).cuda()
+        dy = torch.from_numpy(np.random.default_rng(n + 2).integers(0, 255, size=n, dtype=np.uint8)).cuda()
+        run(x, dy)
+
+
 def test_is_the_relu_backward_of_the_framework_on_a_fused_forward():
     n = 1_000_000 + 3
     x = torch.randn(n, device="cuda", requires_grad=True)
