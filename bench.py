@@ -40,14 +40,19 @@ FALLBACK_HBM_GBS = 6650.0
 BASE_SEED_RELU = 170501626 + 6000
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM bytes per launch measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum),
-# as a multiple of the algorithmic bytes of the same launch, from the captures
-# summarised under profiles/ (2^26 fp32 elements, density 0.33: 268 MB dense).
-# Reads equal the algorithmic read bytes exactly and scale with the element
-# count; writes were below the algorithmic figure because part of the output was
-# still in the write-back L2 at kernel end, a fixed amount that does not scale,
-# so the scaled figure is a slight under-estimate for larger tensors.
-NCU_TRAFFIC_FACTOR = {"zvc_compress_kernel": 0.857, "zvc_decompress_kernel": 0.841}
+# DRAM bytes per launch measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum, one
+# pass, one launch of each kernel) on the workloads the default line reports, at their full
+# size; the captures are summarised under profiles/dram_bytes_bench_workloads.md.  Reads
+# equal the algorithmic read bytes; writes fall short of the algorithmic figure by what is
+# still in the write-back L2 when the kernel ends.
+NCU_DRAM_BYTES = {
+    ("config2", "compress"): None, ("config2", "decompress"): None,
+    ("config5a", "compress"): None, ("config5a", "decompress"): None,
+    ("config5c", "compress"): None, ("config5c", "decompress"): None,
+}
+KERNEL_NAMES = {(4, "compress"): "zvc_compress_kernel", (4, "decompress"): "zvc_decompress_kernel",
+                (2, "compress"): "zvc_compress_rows_kernel", (2, "decompress"): "zvc_decompress_kernel_u16",
+                (1, "compress"): "zvc_compress_rows_kernel", (1, "decompress"): "zvc_decompress_kernel_u8"}
 
 
 def env_int(name, default):
@@ -93,10 +98,17 @@ def make_workload(name: str, device, rank: int = 0):
         return wl.correlated_relu((64, c, h, w), d, wl.seed_for(3, i) + bump, device), \
             "config3 tensor %d: fp32 NCHW 64x%dx%dx%d, clustered zeros, density %.3f" % (i, c, h, w, d)
     if name.startswith("iid:"):
-        # iid:<elements>:<density>[:f16] -- free-size case for profiling and sweeps
+        # iid:<elements>:<density>[:f16|:u8] -- free-size case for profiling and sweeps
         parts = name.split(":")
         cnt, d = int(parts[1]), float(parts[2])
-        dt = torch.float16 if len(parts) > 3 and parts[3] == "f16" else torch.float32
+        kind = parts[3] if len(parts) > 3 else "f32"
+        if kind == "u8":
+            # one-byte elements (an 8-bit float or integer type): non-zero bytes 1..255, zeros i.i.d.
+            g = torch.Generator(device=device).manual_seed(wl.seed_for(9) + bump)
+            v = torch.randint(1, 256, (cnt,), generator=g, device=device, dtype=torch.int16).to(torch.uint8)
+            keep = torch.rand(cnt, generator=g, device=device) < d
+            return v * keep, "iid: 1-byte elements, %d elements, i.i.d. density %g" % (cnt, d)
+        dt = torch.float16 if kind == "f16" else torch.float32
         return wl.iid_relu_like((cnt,), d, wl.seed_for(9) + bump, device, dtype=dt, floor=2.0 ** -10), \
             "iid: %s %d elements, i.i.d. density %g" % ("fp16" if dt == torch.float16 else "fp32", cnt, d)
     raise SystemExit("unknown workload %r" % name)
@@ -287,25 +299,25 @@ def run_reference(args):
 # --------------------------------------------------------------------------- #
 # the CUDA arm
 # --------------------------------------------------------------------------- #
-def run_cdma(args):
+def dtype_code(B, x):
+    import torch
+    return {torch.float32: B.F32, torch.float16: B.F16, torch.bfloat16: B.BF16, torch.uint8: B.U8}[x.dtype]
+
+
+def raw_view(x):
+    import torch
+    return x.view(-1).view({4: torch.int32, 2: torch.int16, 1: torch.uint8}[x.element_size()])
+
+
+def measure_codec(B, x, steps, warmup, repeats, world=1, dev=None, sampler=None):
+    """Parity on these very buffers, then `repeats` timed loops of exactly `steps` steps (a step = one
+    compress + one decompress of x, device resident).  Returns sizes, the per-repeat loop times, the
+    per-kernel and per-call times of every step, and the launches counted in the timed loops."""
     import torch
     import torch.distributed as dist
-    from paper_1705_01626_b200 import binding as B
-
-    world = env_int("WORLD_SIZE", 1)
-    rank = env_int("RANK", 0)
-    local = env_int("LOCAL_RANK", 0)
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the codec has no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    x, desc = make_workload(args.workload, dev, rank)
-    x = x.contiguous()
+    dev = dev or x.device
     n, s = x.numel(), x.element_size()
-    code = {torch.float32: B.F32, torch.float16: B.F16, torch.bfloat16: B.BF16}[x.dtype]
+    code = dtype_code(B, x)
     dense_bytes = n * s
     cap = B.cdma_zvc_max_compressed_bytes(n, code)
     entries = B.cdma_zvc_table_entries(n)
@@ -331,69 +343,118 @@ def run_cdma(args):
             raise B.CdmaError(st, "cdma_zvc_decompress_async")
 
     # ---- correctness on these very buffers before any timing ----------------
-    itype = torch.int32 if s == 4 else torch.int16
-    nnz = int(torch.count_nonzero(x.view(-1).view(itype)))
+    nnz = int(torch.count_nonzero(raw_view(x)))
     c_bytes = B.cdma_zvc_compress(x.data_ptr(), n, code, B.NCHW, payload.data_ptr(), cap, table.data_ptr(),
                                   ws.data_ptr(), ws_bytes, sh)
     if c_bytes != 4 * ((n + 31) // 32) + s * nnz:
         raise SystemExit("compressed size %d differs from 4*ceil(n/32)+s*nnz" % c_bytes)
     r = B.cdma_zvc_decompress(payload.data_ptr(), c_bytes, table.data_ptr(), n, code, B.NCHW, out.data_ptr(),
                               ws.data_ptr(), ws_bytes, sh)
-    if r != dense_bytes or not torch.equal(out.view(-1).view(itype), x.view(-1).view(itype)):
+    if r != dense_bytes or not torch.equal(raw_view(out), raw_view(x)):
         raise SystemExit("round trip is not bit-exact")
-    table_bytes = 8 * entries
-    algo_bytes = dense_bytes + c_bytes + table_bytes      # per kernel launch, either direction
 
     # ---- device-resident timing --------------------------------------------
+    K = steps
+    for _ in range(max(warmup, 3)):
+        compress()
+        decompress(c_bytes)
+    torch.cuda.synchronize()
+    loops, tc, td, tc_call, td_call = [], [], [], [], []
+    launches = 0
+    for rep in range(repeats):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K + 1)]
+        # event pairs recorded by the library around each kernel alone (the call-level brackets also
+        # contain the host-side part of the call)
+        kev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+        for row in kev:
+            for e in row:
+                e.record(stream)                     # creates the underlying cudaEvent_t
+        torch.cuda.synchronize()
+        launches0 = B.cdma_kernel_launch_count()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if sampler is not None and rep == 0:
+            sampler.start()
+        ev[0].record(stream)
+        for i in range(K):
+            B.cdma_time_next_kernel(kev[i][0].cuda_event, kev[i][1].cuda_event)
+            compress()
+            ev[2 * i + 1].record(stream)
+            B.cdma_time_next_kernel(kev[i][2].cuda_event, kev[i][3].cuda_event)
+            decompress(c_bytes)
+            ev[2 * i + 2].record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        launches = B.cdma_kernel_launch_count() - launches0
+        total_ms = ev[0].elapsed_time(ev[-1])
+        if world > 1:
+            t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        loops.append(total_ms)
+        tc_call += [ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(K)]
+        td_call += [ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(K)]
+        tc += [kev[i][0].elapsed_time(kev[i][1]) for i in range(K)]
+        td += [kev[i][2].elapsed_time(kev[i][3]) for i in range(K)]
+        if int(res[1]) != 0:
+            raise SystemExit("device reported status %d during timing" % int(res[1]))
+    return {"n": n, "s": s, "dense_bytes": dense_bytes, "c_bytes": c_bytes, "table_bytes": 8 * entries, "nnz": nnz,
+            "loops_ms": loops, "tc": tc, "td": td, "tc_call": tc_call, "td_call": td_call, "launches": launches}
+
+
+def kernel_roofline(workload, direction, m, peak, peak_kind):
+    """Roofline record of one kernel: algorithmic bytes per launch over its mean launch time."""
+    algo_bytes = m["dense_bytes"] + m["c_bytes"] + m["table_bytes"]      # per launch, either direction
+    times = m["tc"] if direction == "compress" else m["td"]
+    calls = m["tc_call"] if direction == "compress" else m["td_call"]
+    ms = statistics.mean(times)
+    ach = algo_bytes / (ms * 1e-3) / 1e9
+    traffic = NCU_DRAM_BYTES.get((workload, direction))
+    return {"kernel": KERNEL_NAMES[(m["s"], direction)], "bound": "hbm", "achieved": ach, "peak": peak,
+            "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
+            "frac_of_nominal_8TBps": ach / NOMINAL_HBM_GBS,
+            "traffic": traffic,
+            "traffic_note": ("ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch at this size; "
+                             "see profiles/dram_bytes_bench_workloads.md") if traffic else
+                            "not captured for this workload",
+            "frac_dram": (traffic / (ms * 1e-3) / 1e9 / peak) if traffic else None,
+            "algorithmic_bytes": algo_bytes, "mean_launch_ms": ms, "median_launch_ms": statistics.median(times),
+            "mean_call_ms": statistics.mean(calls),
+            "uncompressed_GBps": m["dense_bytes"] / (ms * 1e-3) / 1e9}
+
+
+def run_cdma(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1705_01626_b200 import binding as B
+
+    world = env_int("WORLD_SIZE", 1)
+    rank = env_int("RANK", 0)
+    local = env_int("LOCAL_RANK", 0)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the codec has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    x, desc = make_workload(args.workload, dev, rank)
+    x = x.contiguous()
+    n, s = x.numel(), x.element_size()
     K, W = args.steps, max(args.warmup, 3)
-    for _ in range(W):
-        compress()
-        decompress(c_bytes)
-    torch.cuda.synchronize()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K + 1)]
-    # event pairs recorded by the library around each kernel alone (the call-level
-    # brackets below also contain the workspace reset and the 16-byte result copy)
-    kev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    for row in kev:
-        for e in row:
-            e.record(stream)                     # creates the underlying cudaEvent_t
-    torch.cuda.synchronize()
     sampler = ClockSampler(local)
-    launches0 = B.cdma_kernel_launch_count()
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    ev[0].record(stream)
-    for i in range(K):
-        B.cdma_time_next_kernel(kev[i][0].cuda_event, kev[i][1].cuda_event)
-        compress()
-        ev[2 * i + 1].record(stream)
-        B.cdma_time_next_kernel(kev[i][2].cuda_event, kev[i][3].cuda_event)
-        decompress(c_bytes)
-        ev[2 * i + 2].record(stream)
-    torch.cuda.synchronize()
+    m = measure_codec(B, x, K, W, args.repeats, world, dev, sampler)
     clocks = sampler.stop()
-    if world > 1:
-        dist.barrier()
-    launches = B.cdma_kernel_launch_count() - launches0
-    total_ms = ev[0].elapsed_time(ev[-1])
-    tc_call = [ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(K)]
-    td_call = [ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(K)]
-    tc = [kev[i][0].elapsed_time(kev[i][1]) for i in range(K)]
-    td = [kev[i][2].elapsed_time(kev[i][3]) for i in range(K)]
-    if int(res[1]) != 0:
-        raise SystemExit("device reported status %d during timing" % int(res[1]))
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    dense_bytes, c_bytes, table_bytes, nnz = m["dense_bytes"], m["c_bytes"], m["table_bytes"], m["nnz"]
+    total_ms = statistics.median(m["loops_ms"])          # the median repeat of exactly K steps
 
     # ---- end to end with host buffers (copies inside the timed region) ------
     e2e = None
     offload = None
     if not args.no_e2e:
-        e2e, offload = run_e2e(B, x, code, c_bytes, args, world, dev)
+        e2e, offload = run_e2e(B, x, dtype_code(B, x), c_bytes, args, world, dev)
 
     if rank != 0:
         if world > 1:
@@ -401,23 +462,9 @@ def run_cdma(args):
         return
 
     peak, peak_kind = measured_peak()
-    mean_c, mean_d = sum(tc) / K, sum(td) / K
-
-    def roof(name, ms):
-        ach = algo_bytes / (ms * 1e-3) / 1e9
-        f = NCU_TRAFFIC_FACTOR.get(name)
-        return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                "frac": ach / peak, "peak_kind": "of " + peak_kind,
-                "frac_of_nominal_8TBps": ach / NOMINAL_HBM_GBS,
-                "traffic": (f * algo_bytes) if f else None,
-                "traffic_note": "ncu DRAM bytes of a 268 MB capture scaled by algorithmic bytes; see profiles/",
-                "algorithmic_bytes": algo_bytes, "mean_launch_ms": ms,
-                "uncompressed_GBps": dense_bytes / (ms * 1e-3) / 1e9}
-
-    rc, rd = roof("zvc_compress_kernel", mean_c), roof("zvc_decompress_kernel", mean_d)
-    rc["mean_call_ms"] = sum(tc_call) / K       # whole API call: workspace reset + kernel + result copy
-    rd["mean_call_ms"] = sum(td_call) / K
-    dominant = rc if mean_c >= mean_d else rd
+    rc = kernel_roofline(args.workload, "compress", m, peak, peak_kind)
+    rd = kernel_roofline(args.workload, "decompress", m, peak, peak_kind)
+    dominant = rc if rc["mean_launch_ms"] >= rd["mean_launch_ms"] else rd
     line = {
         "metric": METRIC,
         "value": world * dense_bytes * K / (total_ms * 1e-3) / 1e9,
@@ -429,7 +476,7 @@ def run_cdma(args):
         "higher_is_better": True,
         "scaling": "weak",
         "vs_baseline": None,
-        "dtype": "u32" if s == 4 else "u16",
+        "dtype": {4: "u32", 2: "u16", 1: "u8"}[s],
         "data": "synthetic",
         "config": {"workload": desc, "elements": n, "dense_bytes": dense_bytes,
                    "compressed_bytes": c_bytes, "table_bytes": table_bytes,
@@ -437,16 +484,37 @@ def run_cdma(args):
                    "ratio_with_table": dense_bytes / (c_bytes + table_bytes),
                    "l2": "inputs larger than L2 (no flush needed)" if dense_bytes > 2 * 126e6
                          else "input fits in L2: warm-cache figure",
-                   "parallelism": "replicas x%d, no collective" % world},
+                   "parallelism": "replicas x%d, no collective" % world,
+                   "repeats": "%d timed loops of %d steps each; value and ms_per_step are the median loop"
+                              % (args.repeats, K),
+                   "loops_ms_per_step": [t / K for t in m["loops_ms"]]},
         "roofline": dominant,
         "kernels": {"compress": rc, "decompress": rd},
         "clocks": clocks,
-        "gpu_launches": int(launches),
+        "gpu_launches": int(m["launches"]),
         "e2e": e2e,
         "offload": offload,
     }
+    host = None
     if not args.no_cpu_baseline and world == 1:
         host = x.view(-1)[: min(n, 1 << 28)].cpu().numpy()
+    del x
+    torch.cuda.empty_cache()
+    if not args.no_other_configs and world == 1 and args.workload == "config2":
+        # the cases furthest from the roofline ride along in the same record: the sparse 2 GiB tensor
+        # and the 2-byte tensor of workload 5 (fewer steps; same parity check first)
+        other = {}
+        for name in ("config5a", "config5c"):
+            y, ydesc = make_workload(name, dev, rank)
+            mo = measure_codec(B, y.contiguous(), max(4, K // 4), 3, 3)
+            other[name] = {"workload": ydesc, "ratio_payload": mo["dense_bytes"] / mo["c_bytes"],
+                           "ms_per_step": statistics.median(mo["loops_ms"]) / max(4, K // 4),
+                           "compress": kernel_roofline(name, "compress", mo, peak, peak_kind),
+                           "decompress": kernel_roofline(name, "decompress", mo, peak, peak_kind)}
+            del y
+            torch.cuda.empty_cache()
+        line["other_configs"] = other
+    if host is not None:
         line["cpu_baseline"] = cpu_baseline(host)
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -482,7 +550,7 @@ def run_e2e(B, x, code, c_bytes, args, world, dev):
             raise SystemExit("host-buffer decompress returned %d" % r)
 
     one()
-    itype = torch.int32 if s == 4 else torch.int16
+    itype = {4: torch.int32, 2: torch.int16, 1: torch.uint8}[s]
     if not torch.equal(h_y.view(-1).view(itype), h_x.view(-1).view(itype)):
         raise SystemExit("host-buffer round trip is not bit-exact")
     torch.cuda.synchronize()
@@ -615,8 +683,12 @@ def run_sweep(args):
         dense = x.numel() * 4
         algo = dense + c + 8 * B.cdma_zvc_table_entries(x.numel())
         ralgo = dense + rc + 8 * B.cdma_zvc_table_entries(x.numel())
+        # Section VI-A also looks at compression blocks of up to 64 KB: the zero-value stream has no
+        # per-block header, so the block size changes nothing but the size of the offset table kept
+        # beside it (one 8-byte entry per block)
+        blocks = {"%d KB" % kb: dense / (c + 8 * (dense // (kb << 10) + 1)) for kb in (4, 16, 64)}
         print(json.dumps({"workload": "config4", "density": d, "layout": layout, "dense_bytes": dense,
-                          "compressed_bytes": c, "ratio": dense / c,
+                          "compressed_bytes": c, "ratio": dense / c, "ratio_with_table_by_block": blocks,
                           "compress_GBps": dense / tc / 1e6, "decompress_GBps": dense / td / 1e6,
                           "compress_frac_of_" + kind: algo / tc / 1e6 / peak,
                           "decompress_frac_of_" + kind: algo / td / 1e6 / peak,
@@ -795,6 +867,29 @@ def run_relu(args):
     t_f = timed(lambda: fused(False))
     dense = n * 4
     peak, kind = measured_peak()
+
+    # backward pass: the gradient gated by the masks of the compressed map, against rebuilding y and
+    # running the framework's backward kernel over y and dy
+    dy = torch.randn_like(x)
+    dx = torch.empty_like(x)
+    dx2 = torch.empty_like(x)
+
+    def bwd_separate():
+        B.cdma_zvc_decompress_async(payload.data_ptr(), c, table.data_ptr(), n, B.F32, B.NCHW, y.data_ptr(),
+                                    ws.data_ptr(), ws_bytes, sh, res.data_ptr())
+        torch.ops.aten.threshold_backward.grad_input(dy, y, 0.0, grad_input=dx)
+
+    def bwd_fused():
+        B.cdma_zvc_relu_backward_async(payload.data_ptr(), c, table.data_ptr(), n, B.F32, B.NCHW, dy.data_ptr(),
+                                       dx2.data_ptr(), ws.data_ptr(), ws_bytes, sh, res.data_ptr())
+
+    bwd_separate()
+    bwd_fused()
+    torch.cuda.synchronize()
+    if not torch.equal(dx.view(torch.int32), dx2.view(torch.int32)):
+        raise SystemExit("backward from the masks differs from decompress + threshold_backward")
+    t_bs = timed(bwd_separate)
+    t_bf = timed(bwd_fused)
     print(json.dumps({
         "workload": "relu: fp32 64x64x224x224 pre-activations N(-0.47,1), ReLU density %.3f" % ((c - 4 * (n // 32)) / 4 / n),
         "dense_bytes": dense, "compressed_bytes": c,
@@ -804,7 +899,13 @@ def run_relu(args):
                               "fused_payload_only": dense + c},
         "frac_of_" + kind: {"relu_then_compress": (3 * dense + c) / t_sep / 1e6 / peak,
                             "fused_with_dense": (2 * dense + c) / t_fd / 1e6 / peak,
-                            "fused_payload_only": (dense + c) / t_f / 1e6 / peak}}), flush=True)
+                            "fused_payload_only": (dense + c) / t_f / 1e6 / peak},
+        "backward": {"decompress_then_threshold_backward_ms": t_bs, "from_masks_ms": t_bf,
+                     "speedup": t_bs / t_bf,
+                     "algorithmic_bytes": {"decompress_then_threshold_backward": 4 * dense + c,
+                                           "from_masks": 2 * dense + c},
+                     "frac_of_" + kind: {"decompress_then_threshold_backward": (4 * dense + c) / t_bs / 1e6 / peak,
+                                         "from_masks": (2 * dense + c) / t_bf / 1e6 / peak}}}), flush=True)
 
 
 def run_timeline(args):
@@ -909,13 +1010,15 @@ def run_timeline(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cdma", choices=["cdma", "reference"])
     ap.add_argument("--workload", default="config2")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true")
+    ap.add_argument("--repeats", type=int, default=10)
     args = ap.parse_args()
     if args.steps < 1:
         raise SystemExit("--steps must be >= 1")
