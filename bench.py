@@ -46,9 +46,9 @@ NOMINAL_HBM_GBS = 8000.0
 # equal the algorithmic read bytes; writes fall short of the algorithmic figure by what is
 # still in the write-back L2 when the kernel ends.
 NCU_DRAM_BYTES = {
-    ("config2", "compress"): None, ("config2", "decompress"): None,
-    ("config5a", "compress"): None, ("config5a", "decompress"): None,
-    ("config5c", "compress"): None, ("config5c", "decompress"): None,
+    ("config2", "compress"): 1060378112, ("config2", "decompress"): 1052173824,
+    ("config5a", "compress"): 2312416256, ("config5a", "decompress"): 2263456768,
+    ("config5c", "compress"): 1463992832, ("config5c", "decompress"): 1406410752,
 }
 KERNEL_NAMES = {(4, "compress"): "zvc_compress_kernel", (4, "decompress"): "zvc_decompress_kernel",
                 (2, "compress"): "zvc_compress_rows_kernel", (2, "decompress"): "zvc_decompress_kernel_u16",
