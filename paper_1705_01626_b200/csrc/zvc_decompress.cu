@@ -63,9 +63,11 @@ struct U32Lane {
 // end after every second window, so that nothing is read beyond the staged bytes
 // plus two records; a walk that was pulled back once overshoots again at every
 // later step, so the caller only has to look at the last one.
-template <uint32_t G>
+// GATE: instead of the values of the stream, the elements of `gate` (the incoming gradient of the
+// backward pass) go to the places the masks mark; the values are not even read.
+template <uint32_t G, bool GATE>
 __device__ __forceinline__ void expand_round_u32(uint32_t& a, uint32_t a_end, uint32_t& last, const U32Lane& c,
-                                                 uint4* __restrict__ out) {
+                                                 uint4* __restrict__ out, const uint4* __restrict__ gate) {
     // four serial steps of the self-delimiting walk; every lane sees all four
     const uint32_t a0 = a;
     const uint32_t m0 = lds32<16 * G + 0>(a0);
@@ -79,33 +81,44 @@ __device__ __forceinline__ void expand_round_u32(uint32_t& a, uint32_t a_end, ui
     a = min(last, a_end - (16u * G + 16u));
     const uint32_t my_a = c.w_hi ? (c.w_odd ? a3 : a2) : (c.w_odd ? a1 : a0);
     const uint32_t my_m = c.w_hi ? (c.w_odd ? m3 : m2) : (c.w_odd ? m1 : m0);
+    const uint32_t nib = my_m >> c.sh;
+    const bool b0 = nib & 1u, b1 = nib & 2u, b2 = nib & 4u, b3 = nib & 8u;
+    if (GATE) {
+        (void)my_a;
+        const uint4 g = __ldcs(gate + 32 * G);
+        __stcs(out + 32 * G, make_uint4(b0 ? g.x : 0u, b1 ? g.y : 0u, b2 ? g.z : 0u, b3 ? g.w : 0u));
+        return;
+    }
     // the next four values in front of my elements
     const uint32_t q = my_a + 4u * __popc(my_m & c.below) + c.off;
     const uint32_t v0 = lds32<16 * G + 0>(q), v1 = lds32<16 * G + 4>(q), v2 = lds32<16 * G + 8>(q),
                    v3 = lds32<16 * G + 12>(q);
     // element k takes the value numbered by the set bits below bit k
-    const uint32_t nib = my_m >> c.sh;
-    const bool b0 = nib & 1u, b1 = nib & 2u, b2 = nib & 4u, b3 = nib & 8u;
     const uint32_t t1 = b0 ? v1 : v0, u = b0 ? v2 : v1, w = b0 ? v3 : v2;
     const uint32_t t2 = b1 ? u : t1, x = b1 ? w : u;
     const uint32_t t3 = b2 ? x : t2;
     __stcs(out + 32 * G, make_uint4(b0 ? v0 : 0u, b1 ? t1 : 0u, b2 ? t2 : 0u, b3 ? t3 : 0u));
 }
 
-template <uint32_t G>
+template <uint32_t G, bool GATE>
 __device__ __forceinline__ void expand_rounds_u32(uint32_t& a, uint32_t a_end, uint32_t& last, const U32Lane& c,
-                                                  uint4* __restrict__ out) {
+                                                  uint4* __restrict__ out, const uint4* __restrict__ gate) {
     if constexpr (G < kChunkWindows / 4) {
-        expand_round_u32<G>(a, a_end, last, c, out);
-        expand_rounds_u32<G + 1>(a, a_end, last, c, out);
+        expand_round_u32<G, GATE>(a, a_end, last, c, out, gate);
+        expand_rounds_u32<G + 1, GATE>(a, a_end, last, c, out, gate);
     }
 }
 
-template <typename T, bool PREFETCH>
+// GATE = false: decompression.  GATE = true: the backward pass of the activation function from the
+// compressed map (Section II-B: the backward pass reuses the map; for y = max(x, 0) only its non-zero
+// pattern matters): dst = gate where the map's element is non-zero, else 0 -- the same table checks,
+// staging and walk, but the masks alone are used.
+template <typename T, bool PREFETCH, bool GATE>
 __global__ void __launch_bounds__(kDecThreads, 6)
 zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
                       const uint64_t* __restrict__ table, uint64_t n, T* __restrict__ dst,
-                      uint64_t* __restrict__ ws, const LaunchCtl ctl, uint64_t num_chunks) {
+                      uint64_t* __restrict__ ws, const LaunchCtl ctl, uint64_t num_chunks,
+                      const T* __restrict__ gate) {
     constexpr uint32_t S = sizeof(T);
     constexpr uint32_t MU = 4 / S;                               // units of T per mask
     constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
@@ -202,7 +215,8 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
         c.w_odd = (lane & 8u) != 0u;
         const uint32_t t_addr = static_cast<uint32_t>(__cvta_generic_to_shared(buf));
         uint32_t a = t_addr + 4u * p, last = 0;
-        expand_rounds_u32<0>(a, t_addr + 4u * end, last, c, reinterpret_cast<uint4*>(dst + e0) + lane);
+        expand_rounds_u32<0, GATE>(a, t_addr + 4u * end, last, c, reinterpret_cast<uint4*>(dst + e0) + lane,
+                                   GATE ? reinterpret_cast<const uint4*>(gate + e0) + lane : nullptr);
         // `last` is the final position before it was pulled back, with 4 bytes per window folded out
         p = (last - t_addr) / 4u + kChunkWindows;
     } else {
@@ -218,8 +232,10 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
             const uint32_t left = nelem - w * kWindow;           // elements this window really has
             if (p + MU + cnt > end || (left < kWindow && (m >> left) != 0)) { bad = true; break; }
             const bool bit = (m >> lane) & 1u;
-            const T val = bit ? units[p + MU + __popc(m & lt)] : T(0);
-            if (lane < left) out[w * kWindow] = val;
+            if (lane < left) {
+                const T val = bit ? (GATE ? gate[e0 + lane + w * kWindow] : units[p + MU + __popc(m & lt)]) : T(0);
+                out[w * kWindow] = val;
+            }
             p += MU + cnt;
         }
     }
@@ -442,9 +458,9 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
     if (elem_size == 4) {
         // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
         const bool prefetch = src_on_device && src_bytes >= (n * 4) / 5;
-        auto kernel = prefetch ? zvc_decompress_kernel<uint32_t, true> : zvc_decompress_kernel<uint32_t, false>;
+        auto kernel = prefetch ? zvc_decompress_kernel<uint32_t, true, false> : zvc_decompress_kernel<uint32_t, false, false>;
         kernel<<<grid, kDecThreads, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes, d_table, n,
-                                                 static_cast<uint32_t*>(d_dst), d_ws, ctl, chunks);
+                                                 static_cast<uint32_t*>(d_dst), d_ws, ctl, chunks, nullptr);
     } else {
         const dim3 grid16(static_cast<unsigned>((chunks + kDec16Warps - 1) / kDec16Warps));
         // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
@@ -454,6 +470,22 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
             static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint16_t*>(d_dst),
             d_ws, ctl, chunks);
     }
+    timing_after_launch(stream);
+    count_kernel_launch();
+    return cudaGetLastError();
+}
+
+// Backward gate for 4-byte elements: the decompression kernel with the masks steering the gradient.
+cudaError_t launch_zvc_gate_u32(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                const void* d_gate, void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl,
+                                cudaStream_t stream) {
+    const uint64_t chunks = num_chunks_of(n);
+    if (chunks == 0) return cudaSuccess;
+    const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
+    timing_before_launch(stream);
+    zvc_decompress_kernel<uint32_t, false, true><<<grid, kDecThreads, 0, stream>>>(
+        static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint32_t*>(d_dst), d_ws, ctl, chunks,
+        static_cast<const uint32_t*>(d_gate));
     timing_after_launch(stream);
     count_kernel_launch();
     return cudaGetLastError();
