@@ -117,7 +117,8 @@ uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype);
  *                   bytes below dst_capacity.
  *   d_table         cdma_zvc_table_entries(n) uint64, 8-byte aligned
  *   d_workspace     >= cdma_zvc_workspace_bytes(n, dtype), 16-byte aligned;
- *                   contents on entry are irrelevant
+ *                   contents on entry are irrelevant and nothing is cleared
+ *                   between calls (what a launch reads there carries its tag)
  *   cuda_stream     stream the work is enqueued on
  *
  * cdma_zvc_compress waits for the stream and returns the payload size C
@@ -127,8 +128,8 @@ uint64_t cdma_zvc_workspace_bytes(uint64_t n, int dtype);
  * cdma_zvc_compress_async only enqueues.  h_result must point to two uint64
  * in host memory, 8-byte aligned; once the stream reaches that point
  * h_result[0] holds C and h_result[1] the status code (0 on success).  With
- * page-locked memory (recommended) the two words are stored by a one-warp
- * kernel behind the codec kernel; pageable memory gets a 16-byte copy instead.
+ * page-locked memory (recommended) the codec kernel stores the two words there
+ * itself; pageable memory gets a 16-byte copy behind the kernel instead.
  * d_src, d_dst and d_table may also be device views of page-locked host
  * memory: the kernel then reads / writes over the host link directly.
  */
@@ -176,22 +177,30 @@ int cdma_zvc_relu_compress_async(const void* d_src, uint64_t n, int dtype, int l
  * get offloaded), plug-ins that only ever receive buffers from their host
  * application, start-up and tear-down hooks.  (The paper has no counterpart:
  * its engine needs no software workspace.)  The call takes no workspace; it
- * uses one built into the library, a fixed device array of 1,048,832 bytes that
- * every GPU loading the library holds until the process exits, and it calls no
- * cudaMalloc, cudaFree or any other allocating routine.
+ * uses one built into the library, a fixed device array of 1,048,832 bytes, and
+ * it calls no cudaMalloc, cudaFree or any other allocating routine.
  *
  *   - Serves tensors of at most 2^28 elements; a larger n is refused with
  *     -CDMA_ERR_BUFFER_TOO_SMALL (the built-in workspace is too small for it)
  *     before anything is enqueued.
- *   - The first call made with a given device current looks up the array's
- *     device address on that device (a one-time, synchronous set-up step);
- *     make that first call outside any stream capture.
+ *   - The array belongs to the library's device code: its memory is taken on a
+ *     device when that code is loaded there, which with CUDA's default lazy
+ *     loading is the first call made with that device current (at process start
+ *     with CUDA_MODULE_LOADING=EAGER).  Every call looks up the array's device
+ *     address (a table look-up after the first time).  Make a first call -- one
+ *     with n = 0 will do -- at start-up, while memory is available and outside
+ *     any stream capture; on a device too full to load the code that first call
+ *     returns -CDMA_ERR_OUT_OF_MEMORY.  The memory is held until the process
+ *     exits.
  *   - All calls on a device share the one array, which keeps the previous
- *     call's contents; each call clears the part it uses first.  Two calls
- *     that overlap in time on the same device (different streams or threads)
- *     race on it and give undefined results: serialise them.
- *   - Otherwise identical to cdma_zvc_compress: same arguments and checks, same
- *     payload and table, waits for the stream and returns C or -status.
+ *     call's contents.  Nothing in it has to be cleared: a launch only trusts
+ *     look-back descriptors that carry its own tag and writes its result words
+ *     before reading them.  Two calls that overlap in time on the same device
+ *     (different streams or threads) still race on it and give undefined
+ *     results: serialise them.
+ *   - Otherwise identical to cdma_zvc_compress: same arguments and checks
+ *     (d_src may be a device view of page-locked host memory), same payload and
+ *     table, waits for the stream and returns C or -status.
  */
 int64_t cdma_zvc_compress_static_ws(const void* d_src, uint64_t n, int dtype, int layout,
                                     void* d_dst, uint64_t dst_capacity, uint64_t* d_table,
@@ -418,7 +427,8 @@ int64_t cdma_zvc_decompress_host(cdma_ctx* ctx, const void* h_src, uint64_t src_
 void cdma_time_next_kernel(void* start_event, void* stop_event);
 
 /* Number of kernel launches this library has issued in this process (codec
- * kernels only; memsets and copies are not counted). */
+ * kernels and the copy kernel of cdma_offload_async; copies by the copy engines
+ * are not counted). */
 uint64_t cdma_kernel_launch_count(void);
 
 #ifdef __cplusplus

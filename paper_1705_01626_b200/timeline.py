@@ -80,7 +80,7 @@ def oracle_seconds(layers: Iterable[Layer]) -> float:
 
 
 def summary(layers: Sequence[Layer], pcie_gbs: float, dram_bw_gbs: float = math.inf) -> dict:
-    """Step times and the ratios the paper reports (Fig. 14: performance normalised
+    """Step times and the ratios the paper reports (Fig. 13: performance normalised
     to the oracle; speed-up of compressed over plain copies)."""
     t_oracle = oracle_seconds(layers)
     t_vdnn = step_seconds(layers, pcie_gbs, compressed=False)
