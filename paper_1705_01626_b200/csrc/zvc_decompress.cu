@@ -1,6 +1,7 @@
-// Zero-value decompression (Section V-B, Fig. 10b): the pop-count of a mask
-// tells how many payload values its window takes; values or zeros are steered
-// into the window's 32 places.
+// Zero-value decompression of 4-byte elements (Section V-B, Fig. 10b): the
+// pop-count of a mask tells how many payload values its window takes; values or
+// zeros are steered into the window's 32 places.  (2-byte and 1-byte elements
+// have kernels of their own, in files of their own.)
 //
 // One warp expands one chunk (1024 elements).  The offset table gives the
 // chunk's byte range in the payload; the warp copies that range into shared
@@ -23,29 +24,12 @@ constexpr uint32_t kDecWarps = 8;
 constexpr uint32_t kDecThreads = 32 * kDecWarps;
 constexpr uint32_t kPrefetchAheadCtas = 888;   // 6 CTAs x 148 SMs resident at a time
 
-__device__ __forceinline__ void store4(uint32_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    __stcs(reinterpret_cast<uint4*>(p), make_uint4(a, b, c, d));
-}
-__device__ __forceinline__ void store4(uint16_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    __stcs(reinterpret_cast<uint2*>(p), make_uint2(a | (b << 16), c | (d << 16)));
-}
-
 // Shared-memory loads by 32-bit address + immediate: positions in the staged
 // array are kept as byte addresses so that no index has to be scaled.
 template <uint32_t IMM>
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(IMM));
-    return v;
-}
-__device__ __forceinline__ uint2 lds64(uint32_t addr) {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t v;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(v) : "r"(a), "r"(b), "r"(sel));   // the low 16 bits of sel are used
     return v;
 }
 
@@ -243,203 +227,6 @@ zvc_decompress_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes,
     if (bad && lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
 }
 
-// 2-byte elements.  With half the bytes per element the kernel is bound by
-// instruction issue, not by DRAM, so the staging step spends a little to make
-// the walk and the expansion cheap: the chunk's payload goes to shared memory as
-// an array t[] of 32-bit words, t[k] = the 4 bytes that start at 2-byte unit k
-// (both alignments of every word, twice the bytes).  A mask -- which may start on
-// any 2-byte boundary -- is then ONE shared load, t[p], and so are the two values
-// a lane may need, t[q] = unit q | unit q+1 << 16.  Four windows per round, 8
-// lanes per window; a lane expands 4 consecutive elements: the up-to-4 values it
-// needs are the 8 bytes t[q], t[q+2], and where each goes depends only on the
-// lane's 4 mask bits, so two byte-permute instructions with selectors from a
-// 16-entry table (plus one AND that clears the places of zero elements) do the
-// whole expansion; one 8-byte store per lane, 256 contiguous bytes per warp.
-// Per-lane constants of the 2-byte expansion.
-struct U16Lane {
-    uint32_t sh;         // 4 * (lane & 7): where my 4 mask bits start
-    uint32_t below;      // mask bits of the elements in front of mine
-    uint32_t off;        // 8 * (lane >> 3) + 8: my window's place in the round, past its mask word
-    uint32_t tbl;        // shared address of the expansion table
-    bool w_hi, w_odd;    // bits of lane >> 3
-};
-
-// One round = windows 4G .. 4G+3 of a full chunk.  `a` is the shared byte address
-// of the next mask word in t[] minus 8 bytes per window already passed (a mask is
-// two 2-byte units = two 4-byte entries; folded into the immediates).  The walk is
-// pulled back to the chunk's end after every second window; a walk that was pulled
-// back once overshoots again at every later step, so the caller only looks at `last`.
-template <uint32_t G>
-__device__ __forceinline__ void expand_round_u16(uint32_t& a, uint32_t a_end, uint32_t& last, const U16Lane& c,
-                                                 uint2* __restrict__ out) {
-    // four serial steps of the self-delimiting walk; every lane sees all four
-    const uint32_t a0 = a;
-    const uint32_t m0 = lds32<32 * G + 0>(a0);
-    const uint32_t a1 = a0 + 4u * __popc(m0);
-    const uint32_t m1 = lds32<32 * G + 8>(a1);
-    const uint32_t a2 = min(a1 + 4u * __popc(m1), a_end - (32u * G + 16u));
-    const uint32_t m2 = lds32<32 * G + 16>(a2);
-    const uint32_t a3 = a2 + 4u * __popc(m2);
-    const uint32_t m3 = lds32<32 * G + 24>(a3);
-    last = a3 + 4u * __popc(m3);
-    a = min(last, a_end - (32u * G + 32u));
-    const uint32_t my_a = c.w_hi ? (c.w_odd ? a3 : a2) : (c.w_odd ? a1 : a0);
-    const uint32_t my_m = c.w_hi ? (c.w_odd ? m3 : m2) : (c.w_odd ? m1 : m0);
-    // the next four values in front of my elements: entries q and q + 2
-    const uint32_t q = my_a + 4u * __popc(my_m & c.below) + c.off;
-    const uint32_t v01 = lds32<32 * G + 0>(q), v23 = lds32<32 * G + 8>(q);
-    const uint2 ex = lds64(c.tbl + (((my_m >> c.sh) & 15u) << 3));
-    __stcs(out + 32 * G, make_uint2(prmt(v01, 0u, ex.x), prmt(v01, v23, ex.x >> 16) & ex.y));
-}
-
-template <uint32_t G>
-__device__ __forceinline__ void expand_rounds_u16(uint32_t& a, uint32_t a_end, uint32_t& last, const U16Lane& c,
-                                                  uint2* __restrict__ out) {
-    if constexpr (G < kChunkWindows / 4) {
-        expand_round_u16<G>(a, a_end, last, c, out);
-        expand_rounds_u16<G + 1>(a, a_end, last, c, out);
-    }
-}
-
-constexpr uint32_t kU16MaxUnits = 2 * kChunkWindows + kChunk;          // 1088
-constexpr uint32_t kU16Overrun = 2 * (2 + 32);                         // the walk is pulled back every 2 windows
-constexpr uint32_t kU16Entries = (kU16MaxUnits + 8 + kU16Overrun + 2 + 36 + 7) / 8 * 8;
-// Expansion table of the 2-byte kernel, indexed by a lane's 4 mask bits:
-// {sel0 | sel1 << 16, keep1}.  Element k takes value number popc(bits below k);
-// with v01 / v23 the next four values, elements 0,1 = prmt(v01, 0, sel0) (selector
-// nibble 4 picks a zero byte) and elements 2,3 = prmt(v01, v23, sel1) & keep1.
-__constant__ uint2 kExpandU16[16] = {
-    {0x10104444u, 0x00000000u}, {0x32324410u, 0x00000000u}, {0x32321044u, 0x00000000u}, {0x54543210u, 0x00000000u},
-    {0x32104444u, 0x0000ffffu}, {0x54324410u, 0x0000ffffu}, {0x54321044u, 0x0000ffffu}, {0x76543210u, 0x0000ffffu},
-    {0x10104444u, 0xffff0000u}, {0x32324410u, 0xffff0000u}, {0x32321044u, 0xffff0000u}, {0x54543210u, 0xffff0000u},
-    {0x32104444u, 0xffffffffu}, {0x54324410u, 0xffffffffu}, {0x54321044u, 0xffffffffu}, {0x76543210u, 0xffffffffu},
-};
-
-// t[] takes 4.8 KB per warp, so shared memory allows 46-48 warps per SM; CTAs of 2 warps
-// retire and refill most smoothly (4 warps: 2 % slower, 8 warps: 10 %).
-constexpr uint32_t kDec16Warps = 2;
-constexpr uint32_t kDec16MinCtas = 22;
-constexpr uint32_t kDec16PrefetchCtas = 3256;          // 22 CTAs x 148 SMs resident at a time
-
-template <bool PREFETCH>
-__global__ void __launch_bounds__(32 * kDec16Warps, kDec16MinCtas)
-zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes,
-                          const uint64_t* __restrict__ table, uint64_t n, uint16_t* __restrict__ dst,
-                          uint64_t* __restrict__ ws, const LaunchCtl ctl, uint64_t num_chunks) {
-    constexpr uint32_t S = 2, MU = 2;
-    __shared__ __align__(32) uint32_t s_t[kDec16Warps][kU16Entries];
-    __shared__ uint2 s_expand[16];
-    if (threadIdx.x < 16) s_expand[threadIdx.x] = kExpandU16[threadIdx.x];
-    __syncthreads();
-
-    const uint32_t lane = lane_id();
-    const uint32_t warp = threadIdx.x >> 5;
-    const uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * kDec16Warps + warp;
-    if (blockIdx.x == 0 && threadIdx.x == 0) init_decode_result(ws, ctl, n * S);
-    if (chunk >= num_chunks) return;
-
-    const uint64_t e0 = chunk * kChunk;
-    const uint32_t nelem = (n - e0 < kChunk) ? static_cast<uint32_t>(n - e0) : kChunk;
-    const uint32_t nwin = (nelem + kWindow - 1) / kWindow;
-
-    // ---- the chunk's byte range, validated ----------------------------------
-    const uint64_t lo = __ldg(table + chunk);
-    const uint64_t hi = __ldg(table + chunk + 1);
-    const uint64_t len64 = hi - lo;
-    const uint32_t len = static_cast<uint32_t>(len64);                      // trusted only once len64 is known small
-    bool ok = (lo <= hi) && (hi <= src_bytes) && (len64 <= 4ull * kChunkWindows + 2ull * kChunk) &&
-              (len >= 4u * nwin) && (len <= 4u * nwin + S * nelem) &&
-              (((static_cast<uint32_t>(lo) | len) & 1u) == 0u);
-    if (chunk == 0 && lo != 0) ok = false;
-    if (chunk == num_chunks - 1 && hi != src_bytes) ok = false;
-    if (!ok) {
-        if (lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
-        return;
-    }
-
-    // ---- stage payload bytes [lo, hi) as t[]; t[0] is the word at payload byte a0 ---
-    uint32_t* t = s_t[warp];
-    const uint64_t a0 = lo & ~15ull;
-    const uint32_t span = static_cast<uint32_t>(hi - a0);                  // bytes from a0 to the chunk's end
-    // payload bytes behind a0, as far as this chunk can care (32-bit arithmetic in the loop)
-    const uint32_t avail = (src_bytes - a0 > 8192ull) ? 8192u : static_cast<uint32_t>(src_bytes - a0);
-    const uint8_t* from = src + a0;
-    for (uint32_t off = 16u * lane; off < span; off += 16u * 32u) {
-        uint4 q;
-        uint32_t nxt = 0;                                                  // the unit behind these 16 bytes
-        if (off + 18u <= avail) {
-            q = __ldcs(reinterpret_cast<const uint4*>(from + off));
-            nxt = *reinterpret_cast<const uint16_t*>(from + off + 16);
-        } else {
-            // the payload's last bytes: never read past src_bytes
-            uint32_t wds[4] = {0, 0, 0, 0};
-            for (uint32_t b = 0; b < 16; b += 2) {
-                if (off + b + 2u <= avail) {
-                    const uint32_t h = *reinterpret_cast<const uint16_t*>(from + off + b);
-                    wds[b >> 2] |= h << (8 * (b & 2));
-                }
-            }
-            q = make_uint4(wds[0], wds[1], wds[2], wds[3]);
-        }
-        uint4* row = reinterpret_cast<uint4*>(t + off / 2);                // 8 entries for these 8 units
-        row[0] = make_uint4(q.x, __funnelshift_r(q.x, q.y, 16), q.y, __funnelshift_r(q.y, q.z, 16));
-        row[1] = make_uint4(q.z, __funnelshift_r(q.z, q.w, 16), q.w, __funnelshift_r(q.w, nxt, 16));
-    }
-    if (PREFETCH) {
-        // ask L2 for the payload of the chunk a CTA kDec16PrefetchCtas blocks later will expand
-        // (blocks are dispatched in index order; every line still comes from DRAM once)
-        const uint64_t cf = chunk + static_cast<uint64_t>(kDec16PrefetchCtas) * kDec16Warps;
-        if (cf < num_chunks) {
-            const uint64_t flo = __ldg(table + cf);
-            const uint64_t fhi = __ldg(table + cf + 1);
-            // at most 18 lines of 128 bytes: one per lane
-            const uint64_t line0 = flo & ~127ull;
-            const uint64_t span = fhi - line0;                 // garbage if the entries are bad: checked next
-            if (flo <= fhi && fhi <= src_bytes && span <= 2 * kU16MaxUnits + 127) {
-                if (128u * lane < static_cast<uint32_t>(span))
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src + line0 + 128u * lane));
-            }
-        }
-    }
-    __syncwarp();
-
-    // ---- walk the records and expand ----------------------------------------
-    uint32_t p = static_cast<uint32_t>(lo - a0) / S;        // position in 2-byte units
-    const uint32_t end = span / S;
-    bool bad = false;
-
-    if (nelem == kChunk) {
-        U16Lane c;
-        c.sh = 4u * (lane & 7u);
-        c.below = (1u << c.sh) - 1u;
-        c.off = 8u * (lane >> 3) + 8u;
-        c.tbl = static_cast<uint32_t>(__cvta_generic_to_shared(s_expand));
-        c.w_hi = (lane & 16u) != 0u;
-        c.w_odd = (lane & 8u) != 0u;
-        const uint32_t t_addr = static_cast<uint32_t>(__cvta_generic_to_shared(t));
-        uint32_t a = t_addr + 4u * p, last = 0;
-        expand_rounds_u16<0>(a, t_addr + 4u * end, last, c, reinterpret_cast<uint2*>(dst + e0) + lane);
-        p = (last - t_addr) / 4u + kChunkWindows * MU;   // back to units, the 32 mask words included
-    } else {
-        // ragged last chunk: lane = element, one window per round
-        const uint32_t lt = lanemask_lt();
-        uint16_t* out = dst + e0 + lane;
-        for (uint32_t w = 0; w < nwin; ++w) {
-            if (p + MU > end) { bad = true; break; }
-            const uint32_t m = t[p];
-            const uint32_t cnt = __popc(m);
-            const uint32_t left = nelem - w * kWindow;           // elements this window really has
-            if (p + MU + cnt > end || (left < kWindow && (m >> left) != 0)) { bad = true; break; }
-            const bool bit = (m >> lane) & 1u;
-            const uint16_t val = bit ? static_cast<uint16_t>(t[p + MU + __popc(m & lt)]) : uint16_t(0);
-            if (lane < left) out[w * kWindow] = val;
-            p += MU + cnt;
-        }
-    }
-    if (!bad && p != end) bad = true;
-    if (bad && lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
-}
-
 }  // namespace
 
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
@@ -462,13 +249,8 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
         kernel<<<grid, kDecThreads, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes, d_table, n,
                                                  static_cast<uint32_t*>(d_dst), d_ws, ctl, chunks, nullptr);
     } else {
-        const dim3 grid16(static_cast<unsigned>((chunks + kDec16Warps - 1) / kDec16Warps));
-        // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
-        const bool prefetch = src_on_device && src_bytes >= (n * 2) / 5;
-        auto kernel = prefetch ? zvc_decompress_kernel_u16<true> : zvc_decompress_kernel_u16<false>;
-        kernel<<<grid16, 32 * kDec16Warps, 0, stream>>>(
-            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint16_t*>(d_dst),
-            d_ws, ctl, chunks);
+        const cudaError_t e = launch_zvc_decompress_u16(d_src, src_bytes, d_table, n, d_dst, d_ws, ctl, stream, src_on_device);
+        if (e != cudaSuccess) return e;
     }
     timing_after_launch(stream);
     count_kernel_launch();
