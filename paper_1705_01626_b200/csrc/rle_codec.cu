@@ -43,6 +43,7 @@ rle_compress_kernel(const uint32_t* __restrict__ src, uint64_t n, uint8_t* __res
     const uint32_t lt = lanemask_lt();
     const uint32_t tile = blockIdx.x;          // block-index order, as in the zero-value kernel
     if (tile >= num_tiles) return;
+    if (threadIdx.x == 0) prefetch_future_descriptor(ws, tile, num_tiles);
 
     // ---- load: lane l takes element l of every window; beyond n: zeros -------------
     const uint64_t chunk = static_cast<uint64_t>(tile) * kTileChunks + warp;

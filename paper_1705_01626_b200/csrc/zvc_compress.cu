@@ -239,6 +239,7 @@ zvc_compress_kernel(const T* __restrict__ src, uint64_t n, uint8_t* __restrict__
     const uint32_t tile = blockIdx.x;
     if (tile >= num_tiles) return;
     prefetch_future_tile(src, prefetch_bytes, tile);
+    if (threadIdx.x == 0) prefetch_future_descriptor(ws, tile, num_tiles);
     if ((static_cast<uint64_t>(tile) + 1) * (kTileChunks * kChunk) <= n)
         compress_tile_u32<RELU, true>(src, n, dst, cap, table, ws, ctl, num_tiles, num_chunks, relu_out, tile);
     else
@@ -470,6 +471,7 @@ zvc_compress_kernel_u16(const uint16_t* __restrict__ src, uint64_t n, uint8_t* _
     const uint32_t tile = blockIdx.x;     // block-index order, as in the 4-byte kernel
     if (tile >= num_tiles) return;
     prefetch_future_tile(src, prefetch_bytes, tile);
+    if (threadIdx.x == 0) prefetch_future_descriptor(ws, tile, num_tiles);
     if ((static_cast<uint64_t>(tile) + 1) * (kTileChunksU16 * kChunk) <= n)
         compress_tile_u16<RELU, true>(src, n, dst, cap, table, ws, ctl, num_tiles, num_chunks, relu_out, nan_above, tile);
     else

@@ -161,6 +161,7 @@ zvc_compress_rows_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
     // every thread then fetches its row with plain loads further down)
     if (tid == 0) {
         s_late = 0;
+        prefetch_future_descriptor(ws, tile, num_tiles);
         if (use_tma) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar) : "memory");
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
