@@ -157,6 +157,9 @@ cudaError_t launch_zvc_decompress_u8(const void* d_src, uint64_t src_bytes, cons
 cudaError_t launch_zvc_gate_u32(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
                                 const void* d_gate, void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl,
                                 cudaStream_t stream);
+cudaError_t launch_zvc_gate_u16(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                const void* d_gate, void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl,
+                                cudaStream_t stream);
 cudaError_t launch_zvc_relu_backward(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
                                      uint32_t elem_size, const void* d_dy, void* d_dx, uint64_t* d_ws,
                                      const LaunchCtl& ctl, cudaStream_t stream);

@@ -51,7 +51,7 @@ struct U32Lane {
 // backward pass) go to the places the masks mark; the values are not even read.
 template <uint32_t G, bool GATE>
 __device__ __forceinline__ void expand_round_u32(uint32_t& a, uint32_t a_end, uint32_t& last, const U32Lane& c,
-                                                 uint4* __restrict__ out, const uint4* __restrict__ gate) {
+                                                 uint4* __restrict__ out, const uint4& g) {
     // four serial steps of the self-delimiting walk; every lane sees all four
     const uint32_t a0 = a;
     const uint32_t m0 = lds32<16 * G + 0>(a0);
@@ -69,7 +69,6 @@ __device__ __forceinline__ void expand_round_u32(uint32_t& a, uint32_t a_end, ui
     const bool b0 = nib & 1u, b1 = nib & 2u, b2 = nib & 4u, b3 = nib & 8u;
     if (GATE) {
         (void)my_a;
-        const uint4 g = __ldcs(gate + 32 * G);
         __stcs(out + 32 * G, make_uint4(b0 ? g.x : 0u, b1 ? g.y : 0u, b2 ? g.z : 0u, b3 ? g.w : 0u));
         return;
     }
@@ -87,9 +86,16 @@ __device__ __forceinline__ void expand_round_u32(uint32_t& a, uint32_t a_end, ui
 template <uint32_t G, bool GATE>
 __device__ __forceinline__ void expand_rounds_u32(uint32_t& a, uint32_t a_end, uint32_t& last, const U32Lane& c,
                                                   uint4* __restrict__ out, const uint4* __restrict__ gate) {
+    // four rounds at a time; in the gate form their four loads of the gradient are issued together, in front
     if constexpr (G < kChunkWindows / 4) {
-        expand_round_u32<G, GATE>(a, a_end, last, c, out, gate);
-        expand_rounds_u32<G + 1, GATE>(a, a_end, last, c, out, gate);
+        uint4 g[4];
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) g[i] = GATE ? __ldcs(gate + 32 * (G + i)) : make_uint4(0, 0, 0, 0);
+        expand_round_u32<G + 0, GATE>(a, a_end, last, c, out, g[0]);
+        expand_round_u32<G + 1, GATE>(a, a_end, last, c, out, g[1]);
+        expand_round_u32<G + 2, GATE>(a, a_end, last, c, out, g[2]);
+        expand_round_u32<G + 3, GATE>(a, a_end, last, c, out, g[3]);
+        expand_rounds_u32<G + 4, GATE>(a, a_end, last, c, out, gate);
     }
 }
 

@@ -97,42 +97,62 @@ struct LaneConst {
 // One round = window G of each of the four chunks.  `a` is the shared byte address of the chunk's next mask
 // minus 4 bytes per window already passed (folded into the immediates).  A walk that was pulled back once
 // overshoots again at every later step, so the caller only has to look at `last`.
-template <uint32_t G>
+// GATE: instead of the values of the stream, the elements of `gate` (the incoming gradient of the backward
+// pass) go to the places the masks mark; the values are not even read.
+template <uint32_t G, bool GATE>
 __device__ __forceinline__ void expand_round(uint32_t& a, uint32_t a_end, uint32_t& last, const LaneConst& c,
-                                             uint2* __restrict__ out) {
+                                             uint2* __restrict__ out, const uint2& g) {
     const uint32_t m = prmt(lds16<4 * G>(a), lds16<4 * G + 2>(a), 0x5410u);
     last = a + 2u * __popc(m);
-    // my (up to) four values: 2-byte halves behind the mask
-    const uint32_t q = a + 2u * __popc(m & c.below);
     const uint32_t nib = (m >> c.sh) & 15u;
-    // a lane fetches only as many values as it has non-zero elements: fewer lanes per access, fewer bank conflicts
-    const uint32_t cnt = __popc(nib);
-    const uint32_t v01 = prmt(lds16_if_more<4 * G + 4, 0>(q, cnt), lds16_if_more<4 * G + 6, 1>(q, cnt), 0x5410u);
-    const uint32_t v23 = prmt(lds16_if_more<4 * G + 8, 2>(q, cnt), lds16_if_more<4 * G + 10, 3>(q, cnt), 0x5410u);
-    const uint32_t sel = lds32_at(c.tbl + 4u * nib);
-    // 0xffff where bits 2 / 3 are set: the bits go to the sign positions of two bytes, which a permute replicates
-    const uint32_t x = nib * 0x1020u;
-    const uint32_t keep = prmt(x, x, 0x9988u);
-    __stcs(out + 8 * G, make_uint2(prmt(v01, 0u, sel), prmt(v01, v23, sel >> 16) & keep));
+    // 0xffff where a mask bit is set: the four bits go to the sign positions of the four bytes of x, which a
+    // permute replicates
+    const uint32_t x = nib * 0x10204080u;
+    if (GATE) {
+        __stcs(out + 8 * G, make_uint2(g.x & prmt(x, x, 0x9988u), g.y & prmt(x, x, 0xbbaau)));
+    } else {
+        // my (up to) four values: 2-byte halves behind the mask.  A lane fetches only as many values as it has
+        // non-zero elements: fewer lanes per access, fewer bank conflicts
+        const uint32_t q = a + 2u * __popc(m & c.below);
+        const uint32_t cnt = __popc(nib);
+        const uint32_t v01 = prmt(lds16_if_more<4 * G + 4, 0>(q, cnt), lds16_if_more<4 * G + 6, 1>(q, cnt), 0x5410u);
+        const uint32_t v23 = prmt(lds16_if_more<4 * G + 8, 2>(q, cnt), lds16_if_more<4 * G + 10, 3>(q, cnt), 0x5410u);
+        const uint32_t sel = lds32_at(c.tbl + 4u * nib);
+        __stcs(out + 8 * G, make_uint2(prmt(v01, 0u, sel), prmt(v01, v23, sel >> 16) & prmt(x, x, 0xbbaau)));
+    }
     a = (G & 1u) ? min(last, a_end - 4u * (G + 1u)) : last;
 }
 
-template <uint32_t G>
+// Eight rounds at a time; in the gate form their eight loads of the gradient are issued together, in front.
+template <uint32_t G, bool GATE>
 __device__ __forceinline__ void expand_rounds(uint32_t& a, uint32_t a_end, uint32_t& last, const LaneConst& c,
-                                              uint2* __restrict__ out) {
+                                              uint2* __restrict__ out, const uint2* __restrict__ gate) {
     if constexpr (G < kChunkWindows) {
-        expand_round<G>(a, a_end, last, c, out);
-        expand_rounds<G + 1>(a, a_end, last, c, out);
+        uint2 g[8];
+#pragma unroll
+        for (uint32_t i = 0; i < 8; ++i) g[i] = GATE ? __ldcs(gate + 8 * (G + i)) : make_uint2(0, 0);
+        expand_round<G + 0, GATE>(a, a_end, last, c, out, g[0]);
+        expand_round<G + 1, GATE>(a, a_end, last, c, out, g[1]);
+        expand_round<G + 2, GATE>(a, a_end, last, c, out, g[2]);
+        expand_round<G + 3, GATE>(a, a_end, last, c, out, g[3]);
+        expand_round<G + 4, GATE>(a, a_end, last, c, out, g[4]);
+        expand_round<G + 5, GATE>(a, a_end, last, c, out, g[5]);
+        expand_round<G + 6, GATE>(a, a_end, last, c, out, g[6]);
+        expand_round<G + 7, GATE>(a, a_end, last, c, out, g[7]);
+        expand_rounds<G + 8, GATE>(a, a_end, last, c, out, gate);
     }
 }
 
 // BULK: the group's bytes come in by one bulk copy (the payload lies in device memory); otherwise by the
-// warp's own loads.  PREFETCH: ask L2 for the bytes of the group a later CTA will expand.
-template <bool BULK, bool PREFETCH>
+// warp's own loads.  PREFETCH: ask L2 for the bytes of the group a later CTA will expand.  GATE: the
+// backward pass of the activation function from the compressed map (Section II-B: the backward pass reuses
+// the map; for y = max(x, 0) only its non-zero pattern matters): dst = gate where the map's element is
+// non-zero, else 0 -- the same table checks, staging and walk, but the masks alone are used.
+template <bool BULK, bool PREFETCH, bool GATE>
 __global__ void __launch_bounds__(32, kCtasPerSm)
 zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes, const uint64_t* __restrict__ table,
                           uint64_t n, uint16_t* __restrict__ dst, uint64_t* __restrict__ ws, const LaunchCtl ctl,
-                          uint64_t num_chunks) {
+                          uint64_t num_chunks, const uint16_t* __restrict__ gate) {
     constexpr uint32_t S = 2, MU = 2;
     __shared__ __align__(128) uint8_t s_buf[kBufBytes];
     __shared__ uint32_t s_sel[16];
@@ -250,7 +270,8 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes, c
         c.tbl = sel_addr;
         const uint32_t a_end = buf_addr + static_cast<uint32_t>(hi - a0);
         uint32_t a = buf_addr + static_cast<uint32_t>(lo - a0), last = 0;
-        expand_rounds<0>(a, a_end, last, c, reinterpret_cast<uint2*>(dst + e0) + (lane & 7u));
+        expand_rounds<0, GATE>(a, a_end, last, c, reinterpret_cast<uint2*>(dst + e0) + (lane & 7u),
+                               GATE ? reinterpret_cast<const uint2*>(gate + e0) + (lane & 7u) : nullptr);
         // `last` has 4 bytes per window folded out
         const bool bad = last + 4u * kChunkWindows != a_end;
         if (__any_sync(0xffffffffu, bad) && lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
@@ -276,8 +297,10 @@ zvc_decompress_kernel_u16(const uint8_t* __restrict__ src, uint64_t src_bytes, c
             const uint32_t left = knelem - w * kWindow;           // elements this window really has
             if (p + MU + cnt > end || (left < kWindow && (m >> left) != 0)) { bad = true; break; }
             const bool bit = (m >> lane) & 1u;
-            const uint16_t val = bit ? units[p + MU + __popc(m & lt)] : uint16_t(0);
-            if (lane < left) out[w * kWindow] = val;
+            if (lane < left) {
+                const uint16_t val = bit ? (GATE ? gate[ke0 + lane + w * kWindow] : units[p + MU + __popc(m & lt)]) : uint16_t(0);
+                out[w * kWindow] = val;
+            }
             p += MU + cnt;
         }
         if (!bad && p != end) bad = true;
@@ -295,10 +318,27 @@ cudaError_t launch_zvc_decompress_u16(const void* d_src, uint64_t src_bytes, con
     // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
     const bool prefetch = src_on_device && src_bytes >= (n * 2) / 5;
     const bool bulk = src_on_device && (reinterpret_cast<uintptr_t>(d_src) & 15) == 0;
-    auto kernel = bulk ? (prefetch ? zvc_decompress_kernel_u16<true, true> : zvc_decompress_kernel_u16<true, false>)
-                       : zvc_decompress_kernel_u16<false, false>;
+    auto kernel = bulk ? (prefetch ? zvc_decompress_kernel_u16<true, true, false> : zvc_decompress_kernel_u16<true, false, false>)
+                       : zvc_decompress_kernel_u16<false, false, false>;
     kernel<<<grid, 32, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes, d_table, n,
-                                    static_cast<uint16_t*>(d_dst), d_ws, ctl, chunks);
+                                    static_cast<uint16_t*>(d_dst), d_ws, ctl, chunks, nullptr);
+    return cudaGetLastError();
+}
+
+// Backward gate for 2-byte elements: the decompression kernel with the masks steering the gradient.
+cudaError_t launch_zvc_gate_u16(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                const void* d_gate, void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl,
+                                cudaStream_t stream) {
+    const uint64_t chunks = num_chunks_of(n);
+    if (chunks == 0) return cudaSuccess;
+    const dim3 grid(static_cast<unsigned>((chunks + kQ - 1) / kQ));
+    const bool bulk = !in_host_memory(d_src) && (reinterpret_cast<uintptr_t>(d_src) & 15) == 0;
+    auto kernel = bulk ? zvc_decompress_kernel_u16<true, false, true> : zvc_decompress_kernel_u16<false, false, true>;
+    timing_before_launch(stream);
+    kernel<<<grid, 32, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes, d_table, n,
+                                    static_cast<uint16_t*>(d_dst), d_ws, ctl, chunks, static_cast<const uint16_t*>(d_gate));
+    timing_after_launch(stream);
+    count_kernel_launch();
     return cudaGetLastError();
 }
 

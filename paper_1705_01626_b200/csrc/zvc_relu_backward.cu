@@ -10,8 +10,8 @@
 // traffic instead of the 4 n s + C of decompressing y and then running the
 // framework's backward kernel over y and dy.
 //
-// This file holds the kernel for 2-byte and 1-byte elements; 4-byte elements use the decompression
-// kernel of zvc_decompress.cu in its gate form.
+// This file holds the kernel for 1-byte elements; 4-byte and 2-byte elements use the decompression
+// kernels of zvc_decompress.cu and zvc_decompress_u16.cu in their gate form.
 //
 // One warp per chunk.  The chunk's payload lines are first pulled into L1 by one
 // load per lane, all in flight together; the self-delimiting walk from mask to mask
@@ -159,18 +159,14 @@ cudaError_t launch_zvc_relu_backward(const void* d_src, uint64_t src_bytes, cons
                                      const LaunchCtl& ctl, cudaStream_t stream) {
     const uint64_t chunks = num_chunks_of(n);
     if (chunks == 0) return cudaSuccess;
-    // 4-byte elements take the decompression kernel in its gate form (shared-memory staging, the tuned walk)
+    // 4-byte and 2-byte elements take their decompression kernel in its gate form (staging, the tuned walk)
     if (elem_size == 4) return launch_zvc_gate_u32(d_src, src_bytes, d_table, n, d_dy, d_dx, d_ws, ctl, stream);
+    if (elem_size == 2) return launch_zvc_gate_u16(d_src, src_bytes, d_table, n, d_dy, d_dx, d_ws, ctl, stream);
     const dim3 grid(static_cast<unsigned>((chunks + kBwdWarps - 1) / kBwdWarps));
     timing_before_launch(stream);
-    if (elem_size == 2)
-        zvc_relu_backward_kernel<2><<<grid, 32 * kBwdWarps, 0, stream>>>(
-            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<const uint8_t*>(d_dy),
-            static_cast<uint8_t*>(d_dx), d_ws, ctl, chunks);
-    else
-        zvc_relu_backward_kernel<1><<<grid, 32 * kBwdWarps, 0, stream>>>(
-            static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<const uint8_t*>(d_dy),
-            static_cast<uint8_t*>(d_dx), d_ws, ctl, chunks);
+    zvc_relu_backward_kernel<1><<<grid, 32 * kBwdWarps, 0, stream>>>(
+        static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<const uint8_t*>(d_dy),
+        static_cast<uint8_t*>(d_dx), d_ws, ctl, chunks);
     timing_after_launch(stream);
     count_kernel_launch();
     return cudaGetLastError();
