@@ -51,8 +51,8 @@ NCU_DRAM_BYTES = {
     ("config5c", "compress"): 1463992832, ("config5c", "decompress"): 1406410752,
 }
 KERNEL_NAMES = {(4, "compress"): "zvc_compress_kernel", (4, "decompress"): "zvc_decompress_kernel",
-                (2, "compress"): "zvc_compress_rows_kernel", (2, "decompress"): "zvc_decompress_kernel_u16",
-                (1, "compress"): "zvc_compress_rows_kernel", (1, "decompress"): "zvc_decompress_kernel_u8"}
+                (2, "compress"): "zvc_compress_rows_kernel", (2, "decompress"): "zvc_decompress_groups_kernel",
+                (1, "compress"): "zvc_compress_rows_kernel", (1, "decompress"): "zvc_decompress_groups_kernel"}
 
 
 def env_int(name, default):

@@ -149,17 +149,16 @@ cudaError_t launch_zvc_relu_compress(const void* d_src, uint64_t n, uint32_t ele
 cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const uint64_t* d_table,
                                   uint64_t n, uint32_t elem_size, void* d_dst, uint64_t* d_ws,
                                   const LaunchCtl& ctl, cudaStream_t stream, bool src_on_device = true);
-cudaError_t launch_zvc_decompress_u16(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
-                                      void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream,
-                                      bool src_on_device);
-cudaError_t launch_zvc_decompress_u8(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
-                                     void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream);
+// 2-byte and 1-byte elements (zvc_decompress_groups.cu); the caller brackets the launch with the timing hooks
+cudaError_t launch_zvc_decompress_groups(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                         uint32_t elem_size, void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl,
+                                         cudaStream_t stream, bool src_on_device);
 cudaError_t launch_zvc_gate_u32(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
                                 const void* d_gate, void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl,
                                 cudaStream_t stream);
-cudaError_t launch_zvc_gate_u16(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
-                                const void* d_gate, void* d_dst, uint64_t* d_ws, const LaunchCtl& ctl,
-                                cudaStream_t stream);
+cudaError_t launch_zvc_gate_groups(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                   uint32_t elem_size, const void* d_gate, void* d_dst, uint64_t* d_ws,
+                                   const LaunchCtl& ctl, cudaStream_t stream);
 cudaError_t launch_zvc_relu_backward(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
                                      uint32_t elem_size, const void* d_dy, void* d_dx, uint64_t* d_ws,
                                      const LaunchCtl& ctl, cudaStream_t stream);

@@ -1,7 +1,7 @@
 // Zero-value decompression of 4-byte elements (Section V-B, Fig. 10b): the
 // pop-count of a mask tells how many payload values its window takes; values or
 // zeros are steered into the window's 32 places.  (2-byte and 1-byte elements
-// have kernels of their own, in files of their own.)
+// have a kernel of their own, in zvc_decompress_groups.cu.)
 //
 // One warp expands one chunk (1024 elements).  The offset table gives the
 // chunk's byte range in the payload; the warp copies that range into shared
@@ -242,12 +242,6 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
     if (chunks == 0) return cudaSuccess;
     const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
     timing_before_launch(stream);
-    if (elem_size == 1) {
-        const cudaError_t e = launch_zvc_decompress_u8(d_src, src_bytes, d_table, n, d_dst, d_ws, ctl, stream);
-        timing_after_launch(stream);
-        count_kernel_launch();
-        return e;
-    }
     if (elem_size == 4) {
         // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
         const bool prefetch = src_on_device && src_bytes >= (n * 4) / 5;
@@ -255,7 +249,8 @@ cudaError_t launch_zvc_decompress(const void* d_src, uint64_t src_bytes, const u
         kernel<<<grid, kDecThreads, 0, stream>>>(static_cast<const uint8_t*>(d_src), src_bytes, d_table, n,
                                                  static_cast<uint32_t*>(d_dst), d_ws, ctl, chunks, nullptr);
     } else {
-        const cudaError_t e = launch_zvc_decompress_u16(d_src, src_bytes, d_table, n, d_dst, d_ws, ctl, stream, src_on_device);
+        const cudaError_t e = launch_zvc_decompress_groups(d_src, src_bytes, d_table, n, elem_size, d_dst, d_ws, ctl,
+                                                           stream, src_on_device);
         if (e != cudaSuccess) return e;
     }
     timing_after_launch(stream);
@@ -277,6 +272,15 @@ cudaError_t launch_zvc_gate_u32(const void* d_src, uint64_t src_bytes, const uin
     timing_after_launch(stream);
     count_kernel_launch();
     return cudaGetLastError();
+}
+
+// The backward pass of the activation function straight from the compressed map: every element width takes
+// its decompression kernel in the gate form.
+cudaError_t launch_zvc_relu_backward(const void* d_src, uint64_t src_bytes, const uint64_t* d_table, uint64_t n,
+                                     uint32_t elem_size, const void* d_dy, void* d_dx, uint64_t* d_ws,
+                                     const LaunchCtl& ctl, cudaStream_t stream) {
+    if (elem_size == 4) return launch_zvc_gate_u32(d_src, src_bytes, d_table, n, d_dy, d_dx, d_ws, ctl, stream);
+    return launch_zvc_gate_groups(d_src, src_bytes, d_table, n, elem_size, d_dy, d_dx, d_ws, ctl, stream);
 }
 
 }  // namespace cdma
