@@ -26,16 +26,6 @@ namespace cdma {
 
 namespace {
 
-// Four consecutive elements as zero-extended 32-bit values.
-__device__ __forceinline__ void load4(const uint32_t* p, uint32_t (&e)[4]) {
-    const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
-    e[0] = q.x; e[1] = q.y; e[2] = q.z; e[3] = q.w;
-}
-__device__ __forceinline__ void load4(const uint16_t* p, uint32_t (&e)[4]) {
-    const uint2 q = __ldcs(reinterpret_cast<const uint2*>(p));
-    e[0] = q.x & 0xffffu; e[1] = q.x >> 16; e[2] = q.y & 0xffffu; e[3] = q.y >> 16;
-}
-
 // Tiles follow the block index and blocks are dispatched in that order, so the
 // tile `kPrefetchAhead` places further on will be picked up by a CTA that starts
 // about half a CTA lifetime from now (5 CTAs x 148 SMs are resident at a time).

@@ -144,6 +144,42 @@ def test_host_buffer_calls_match_the_oracle(dtype, pinned):
         B.cdma_ctx_destroy(ctx)
 
 
+def test_one_byte_elements_through_the_pipeline_and_the_host_buffer_calls():
+    """1-byte elements: staged offload / prefetch, direct offload / prefetch, and the page-locked
+    host-buffer calls (kernels reading and writing host memory), all against the oracle."""
+    n = 900_000 + 41
+    raw = np.random.default_rng(12).integers(1, 255, size=n, dtype=np.uint8)
+    raw[np.random.default_rng(13).random(n) >= 0.35] = 0
+    x = torch.from_numpy(raw).cuda()
+    want, want_table = zvc_c.compress(raw)
+    cap = B.cdma_zvc_max_compressed_bytes(n, B.U8)
+    entries = B.cdma_zvc_table_entries(n)
+    ctx = B.cdma_ctx_create(4 * (cap + 8 * entries + 4096), 2 * (cap + 8 * entries + B.cdma_zvc_workspace_bytes(n, B.U8) + 4096))
+    try:
+        for offload, prefetch in ((B.cdma_offload, B.cdma_prefetch), (B.cdma_offload_direct, B.cdma_prefetch_direct)):
+            c, ticket = offload(ctx, x.data_ptr(), n, B.U8, B.NCHW, 0)
+            assert c == len(want), B.status_string(c)
+            assert B.cdma_ctx_synchronize(ctx) == 0
+            payload, table = host_view(ctx, ticket, c, entries)
+            assert payload.tobytes() == want.tobytes()
+            assert np.array_equal(table, want_table)
+            out = torch.full_like(x, 7)
+            assert prefetch(ctx, ticket, out.data_ptr(), 0) == n
+            assert torch.equal(out, x)
+        h_x = torch.from_numpy(raw).pin_memory()
+        h_p = torch.zeros(cap, dtype=torch.uint8).pin_memory()
+        h_t = torch.zeros(entries, dtype=torch.int64).pin_memory()
+        h_y = torch.zeros(n, dtype=torch.uint8).pin_memory()
+        c = B.cdma_zvc_compress_host(ctx, h_x.data_ptr(), n, B.U8, B.NCHW, h_p.data_ptr(), cap, h_t.data_ptr())
+        assert c == len(want), B.status_string(c)
+        assert h_p[:c].numpy().tobytes() == want.tobytes()
+        assert np.array_equal(h_t.numpy().view(np.uint64), want_table)
+        assert B.cdma_zvc_decompress_host(ctx, h_p.data_ptr(), c, h_t.data_ptr(), n, B.U8, B.NCHW, h_y.data_ptr()) == n
+        assert torch.equal(h_y, h_x)
+    finally:
+        B.cdma_ctx_destroy(ctx)
+
+
 def host_view(ctx, ticket, nbytes, entries):
     st, hp, ht = B.cdma_ticket_host_view(ctx, ticket)
     assert st == 0

@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from oracle import relu_backward as rb
-from oracle import zvc_c
+from oracle import zvc_c, zvc_numpy
 from paper_1705_01626_b200 import binding as B
 from paper_1705_01626_b200 import workloads as wl
 from tests.gpu_helpers import DT, DeviceCodec, raw_numpy
@@ -70,26 +70,38 @@ def test_in_place_and_special_values():
     run(h, wl.special_values(70_001, seed=9, dtype=torch.float16, device="cuda"))
 
 
-def test_corrupt_streams_and_bad_arguments_are_refused():
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.uint8])
+def test_corrupt_streams_and_bad_arguments_are_refused(dtype):
     n = 20_000
-    x = wl.iid_relu_like((n,), 0.4, seed=77, device="cuda")
-    dy = torch.randn(n, device="cuda")
+    s = torch.empty(0, dtype=dtype).element_size()
+    if dtype == torch.uint8:
+        raw = np.random.default_rng(5).integers(1, 255, size=n, dtype=np.uint8)
+        raw[np.random.default_rng(6).random(n) >= 0.4] = 0
+        x = torch.from_numpy(raw).cuda()
+        dy = torch.from_numpy(np.random.default_rng(7).integers(0, 255, size=n, dtype=np.uint8)).cuda()
+    else:
+        x = wl.iid_relu_like((n,), 0.4, seed=77, device="cuda", dtype=dtype, floor=2.0 ** -10)
+        dy = torch.randn(n, device="cuda").to(dtype)
     dx = torch.empty_like(dy)
-    codec = DeviceCodec(n, torch.float32)
+    codec = DeviceCodec(n, dtype)
     c = codec.compress(x)
     args = lambda payload_bytes=c, table=codec.table: (codec.payload.data_ptr(), payload_bytes, table.data_ptr(), n,
-                                                       B.F32, B.NCHW, dy.data_ptr(), dx.data_ptr(),
+                                                       codec.code, B.NCHW, dy.data_ptr(), dx.data_ptr(),
                                                        codec.ws.data_ptr(), codec.ws_bytes, 0)
     bad = codec.table.clone()
     bad[3] += 4
     assert B.cdma_zvc_relu_backward(*args(table=bad)) == -B.ERR_CORRUPT_STREAM
     assert B.cdma_zvc_relu_backward(*args(payload_bytes=c - 4)) == -B.ERR_CORRUPT_STREAM
     payload = codec.payload.clone()
-    codec.payload[int(codec.table[2])] ^= 0x10                        # one mask bit flipped: the walk misses the chunk's end
+    # one bit flipped in the mask of a chunk's last window: the walk misses the chunk's end
+    # (an earlier window could fall back into step on narrow elements)
+    last_mask = int(zvc_numpy.window_offsets(raw_numpy(x))[3 * 32 - 1])
+    codec.payload[last_mask] ^= 0x10
     assert B.cdma_zvc_relu_backward(*args()) == -B.ERR_CORRUPT_STREAM
     codec.payload.copy_(payload)
-    assert B.cdma_zvc_relu_backward(*args()) == 4 * n                  # and the intact stream still works
+    assert B.cdma_zvc_relu_backward(*args()) == s * n                  # and the intact stream still works
+    assert codec.canaries_intact()
     # overlap of dx with the payload
-    assert B.cdma_zvc_relu_backward(codec.payload.data_ptr(), c, codec.table.data_ptr(), n, B.F32, B.NCHW,
+    assert B.cdma_zvc_relu_backward(codec.payload.data_ptr(), c, codec.table.data_ptr(), n, codec.code, B.NCHW,
                                     dy.data_ptr(), codec.payload.data_ptr(), codec.ws.data_ptr(), codec.ws_bytes,
                                     0) == -B.ERR_INVALID_ARG
