@@ -18,6 +18,7 @@ pytestmark = pytest.mark.gpu
 
 TILE = 8 * 1024      # elements one CTA compresses (4-byte elements; twice that for 2-byte)
 SIZES = [0, 1, 31, 32, 33, 63, 64, 65, 1023, 1024, 1025, 2047, 2048, 2049,
+         3072, 4095, 4096, 4097, 5120,        # around the four-chunk groups of the narrow-element decoder
          TILE - 1, TILE, TILE + 1, 32 * 1024 - 1, 32 * 1024 + 1,
          5 * TILE + 1024 + 17, 40 * TILE + 999]
 
