@@ -21,7 +21,7 @@ CORES = len(os.sched_getaffinity(0))
 
 
 def bits(x):
-    return x.view(-1).view(torch.int32 if x.element_size() == 4 else torch.int16)
+    return x.view(-1).view({4: torch.int32, 2: torch.int16, 1: torch.uint8}[x.element_size()])
 
 
 def full_compare(x):
@@ -163,3 +163,18 @@ def test_config3_offload_set_full_size(mode):
         B.cdma_ctx_destroy(ctx)
         del tensors
         torch.cuda.empty_cache()
+
+
+def test_more_than_two_to_the_32_elements():
+    """Element indices beyond 32 bits: 2^32 + 70,001 one-byte elements (4 GiB; ragged chunk, group and tile),
+    the whole payload and table against the oracle, and the round trip."""
+    n = (1 << 32) + 70_001
+    g = torch.Generator(device="cuda").manual_seed(170501626 + 5900)
+    x = torch.randint(1, 256, (n,), dtype=torch.uint8, device="cuda", generator=g)
+    # zeros in runs of 1 .. 4096 elements so that chunks differ widely in size
+    keep = torch.rand((n + 4095) // 4096, device="cuda", generator=g) < 0.3
+    x *= keep.repeat_interleave(4096)[:n].to(torch.uint8)
+    x *= (torch.rand(n, device="cuda", generator=g) < 0.8).to(torch.uint8)
+    del keep
+    c = full_compare(x)
+    assert c == 4 * ((n + 31) // 32) + int(torch.count_nonzero(x))
