@@ -5,12 +5,14 @@
 // With fewer bytes per element, these widths are bound by the instructions and the
 // shared-memory accesses spent per chunk, not by DRAM.  Three choices keep both low:
 //
-//   - A warp expands four consecutive chunks at once, eight lanes per chunk.  The
-//     walk from mask to mask (the stream is self-delimiting, Section V-A) is serial
-//     within a chunk and every lane of a warp repeats it, so its instructions cost
-//     the same whatever the lanes hold: one walk step now advances four chunks.  A
-//     lane's window is simply the one its group of eight lanes has just reached.
-//   - The four chunks are one contiguous piece of the payload.  One bulk copy
+//   - A warp expands several consecutive chunks at once: four chunks of 2-byte
+//     elements (eight lanes per chunk) or eight chunks of 1-byte elements (four
+//     lanes per chunk).  The walk from mask to mask (the stream is self-delimiting,
+//     Section V-A) is serial within a chunk and every lane of a warp repeats it, so
+//     its instructions cost the same whatever the lanes hold: one walk step now
+//     advances all the warp's chunks.  A lane's window is simply the one its group
+//     of lanes has just reached.
+//   - Those chunks are one contiguous piece of the payload.  One bulk copy
 //     (cp.async.bulk, completion on an mbarrier) brings it into shared memory: no
 //     load or store instruction of the warp is spent on staging.  Masks and values
 //     sit at element boundaries there: 2-byte elements are read as 2-byte halves,
@@ -18,10 +20,11 @@
 //   - A lane fetches only as many values as it has non-zero elements (predicated
 //     loads): fewer lanes per access, fewer bank conflicts between the four chunks.
 //
-// A lane expands 4 consecutive elements: the pop-count of the mask bits below them
-// is where its values start, and byte permutes with selectors from a 16-entry
-// table (indexed by the lane's 4 mask bits) put values and zeros in place; one
-// store per lane, 64 (32) contiguous bytes per chunk and round.  The table and
+// A lane expands 8 bytes of the tensor per round (4 two-byte or 8 one-byte
+// elements): the pop-count of the mask bits below them is where its values start,
+// and byte permutes with selectors from a 16-entry table (indexed by 4 mask bits)
+// put values and zeros in place; one 8-byte store per lane, a window's 64 or 32
+// bytes contiguous.  The table and
 // every record are validated; nothing is read outside the payload or written
 // outside the tensor whatever the input holds.
 //
@@ -37,18 +40,21 @@ namespace cdma {
 
 namespace {
 
-constexpr uint32_t kQ = 4;                                              // chunks per warp
-constexpr uint32_t kLanesPerChunk = 32 / kQ;
 constexpr uint32_t kTryWaitHintNs = 100000;
 
 // Sizes by element width S.
 template <uint32_t S>
 struct Geometry {
+    // a lane expands 8 bytes of the tensor per round: 4 two-byte or 8 one-byte elements; a window takes 8 or 4
+    // lanes, so a warp walks 4 or 8 chunks at once
+    static constexpr uint32_t kLaneElems = 8 / S;
+    static constexpr uint32_t kLanesPerChunk = kWindow / kLaneElems;
+    static constexpr uint32_t kQ = 32 / kLanesPerChunk;                  // chunks per warp
     static constexpr uint32_t kMaxChunkBytes = 4 * kChunkWindows + S * kChunk;
     // The walk is pulled back to the chunk's end after every second window, so it can run two records past
     // it, and a lane reads a mask and up to 4 values (two words) from there.
     static constexpr uint32_t kOverrunBytes = 2 * (4 + S * kWindow);
-    static constexpr uint32_t kBufBytes = (16 + kQ * kMaxChunkBytes + kOverrunBytes + 4 + S * 36 + 8 + 15) / 16 * 16;
+    static constexpr uint32_t kBufBytes = (16 + kQ * kMaxChunkBytes + kOverrunBytes + 4 + S * 36 + 16 + 15) / 16 * 16;
     // CTAs of one warp: what shared memory allows, at most 32
     static constexpr uint32_t kCtasBySmem = (227u * 1024u) / (kBufBytes + 1024u + 128u);
     static constexpr uint32_t kCtasPerSm = kCtasBySmem > 32 ? 32 : kCtasBySmem;
@@ -123,20 +129,18 @@ __device__ __forceinline__ bool wait_copy(uint32_t mbar, uint64_t limit_ns) {
 }
 
 struct LaneConst {
-    uint32_t sh;         // 4 * (lane & 7): where my 4 mask bits start
+    uint32_t sh;         // where my 4 (8) mask bits start
     uint32_t below;      // mask bits of the elements in front of mine
     uint32_t tbl;        // shared address of the selector table
 };
 
-// One round = window G of each of the four chunks.  `a` is the shared byte address of the chunk's next mask
+// One round = window G of each of the warp's chunks.  `a` is the shared byte address of the chunk's next mask
 // minus 4 bytes per window already passed (folded into the immediates).  A walk that was pulled back once
 // overshoots again at every later step, so the caller only has to look at `last`.
-// A lane's share of one round: 8 bytes (2-byte elements) or 4 bytes (1-byte elements).
-template <uint32_t S> struct LaneWord;
-template <> struct LaneWord<2> { using type = uint2; };
-template <> struct LaneWord<1> { using type = uint32_t; };
+// A lane's share of one round: 8 bytes (4 two-byte or 8 one-byte elements).
+template <uint32_t S> struct LaneWord { using type = uint2; };
 
-// One round = window G of each of the four chunks.  `a` is the shared byte address of the chunk's next mask
+// One round = window G of each of the warp's chunks.  `a` is the shared byte address of the chunk's next mask
 // minus 4 bytes per window already passed (folded into the immediates).  A walk that was pulled back once
 // overshoots again at every later step, so the caller only has to look at `last`.
 // GATE: instead of the values of the stream, the elements of `gate` (the incoming gradient of the backward
@@ -171,18 +175,24 @@ __device__ __forceinline__ void expand_round(uint32_t& a, uint32_t a_end, uint32
             __stcs(out + 8 * G, make_uint2(prmt(v01, 0u, sel), prmt(v01, v23, sel >> 16) & prmt(x, x, 0xbbaau)));
         }
     } else {
+        // eight elements: two groups of four, the second group's values right behind the first's
+        const uint32_t nib_hi = (m >> (c.sh + 4u)) & 15u;
+        const uint32_t x_hi = nib_hi * 0x10204080u;
         if (GATE) {
-            __stcs(out + 8 * G, g & prmt(x, x, 0xba98u));
+            __stcs(out + 4 * G, make_uint2(g.x & prmt(x, x, 0xba98u), g.y & prmt(x_hi, x_hi, 0xba98u)));
         } else {
-            // my (up to) four values: the bytes behind the mask, from the aligned word they start in and, when
-            // they reach past it, the next one
+            // my (up to) eight values: the bytes behind the mask, from the aligned word they start in and, as far
+            // as they reach, the next two
             const uint32_t q = a + __popc(m & c.below);
             const uint32_t qa = q & ~3u, ph = q & 3u;
-            const uint32_t cnt = __popc(nib);
-            const uint32_t w0 = lds32_if_more<4 * G + 4, 0>(qa, cnt);
-            const uint32_t w1 = lds32_if_more<4 * G + 8, 4>(qa, ph + cnt);
-            const uint32_t sel = lds32_at(c.tbl + 4u * nib);
-            __stcs(out + 8 * G, prmt(__funnelshift_r(w0, w1, 8u * ph), 0u, sel));
+            const uint32_t c0 = __popc(nib);
+            const uint32_t reach = ph + c0 + __popc(nib_hi);
+            const uint32_t w0 = lds32_if_more<4 * G + 4, 0>(qa, reach - ph);
+            const uint32_t w1 = lds32_if_more<4 * G + 8, 4>(qa, reach);
+            const uint32_t w2 = lds32_if_more<4 * G + 12, 8>(qa, reach);
+            const uint32_t v_lo = __funnelshift_r(w0, w1, 8u * ph), v_hi = __funnelshift_r(w1, w2, 8u * ph);
+            const uint32_t sel_lo = lds32_at(c.tbl + 4u * nib), sel_hi = lds32_at(c.tbl + 4u * nib_hi);
+            __stcs(out + 4 * G, make_uint2(prmt(v_lo, 0u, sel_lo), prmt(__funnelshift_rc(v_lo, v_hi, 8u * c0), 0u, sel_hi)));
         }
     }
     a = (G & 1u) ? min(last, a_end - 4u * (G + 1u)) : last;
@@ -196,7 +206,8 @@ __device__ __forceinline__ void expand_rounds(uint32_t& a, uint32_t a_end, uint3
     if constexpr (G < kChunkWindows) {
         typename LaneWord<S>::type g[8];
 #pragma unroll
-        for (uint32_t i = 0; i < 8; ++i) g[i] = GATE ? __ldcs(gate + 8 * (G + i)) : typename LaneWord<S>::type{};
+        for (uint32_t i = 0; i < 8; ++i)
+            g[i] = GATE ? __ldcs(gate + Geometry<S>::kLanesPerChunk * (G + i)) : typename LaneWord<S>::type{};
         expand_round<S, G + 0, GATE>(a, a_end, last, c, out, g[0]);
         expand_round<S, G + 1, GATE>(a, a_end, last, c, out, g[1]);
         expand_round<S, G + 2, GATE>(a, a_end, last, c, out, g[2]);
@@ -218,6 +229,8 @@ zvc_decompress_groups_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes
                              uint64_t n, uint8_t* __restrict__ dst, uint64_t* __restrict__ ws, const LaunchCtl ctl,
                              uint64_t num_chunks, const uint8_t* __restrict__ gate) {
     using Word = typename LaneWord<S>::type;
+    constexpr uint32_t kQ = Geometry<S>::kQ;
+    constexpr uint32_t kLanesPerChunk = Geometry<S>::kLanesPerChunk;
     constexpr uint32_t kMaxChunkBytes = Geometry<S>::kMaxChunkBytes;
     constexpr uint32_t kBufBytes = Geometry<S>::kBufBytes;
     constexpr uint32_t kPrefetchGroups = Geometry<S>::kPrefetchGroups;
@@ -328,13 +341,13 @@ zvc_decompress_groups_kernel(const uint8_t* __restrict__ src, uint64_t src_bytes
     if (nchunks == kQ && n - c0 * kChunk >= kQ * kChunk) {
         // four full chunks: every group of eight lanes walks its own chunk
         LaneConst c;
-        c.sh = 4u * (lane & 7u);
+        c.sh = Geometry<S>::kLaneElems * (lane % kLanesPerChunk);
         c.below = (1u << c.sh) - 1u;
         c.tbl = sel_addr;
         const uint32_t a_end = buf_addr + static_cast<uint32_t>(hi - a0);
         uint32_t a = buf_addr + static_cast<uint32_t>(lo - a0), last = 0;
-        expand_rounds<S, 0, GATE>(a, a_end, last, c, reinterpret_cast<Word*>(dst + e0 * S) + (lane & 7u),
-                                  GATE ? reinterpret_cast<const Word*>(gate + e0 * S) + (lane & 7u) : nullptr);
+        expand_rounds<S, 0, GATE>(a, a_end, last, c, reinterpret_cast<Word*>(dst + e0 * S) + (lane % kLanesPerChunk),
+                                  GATE ? reinterpret_cast<const Word*>(gate + e0 * S) + (lane % kLanesPerChunk) : nullptr);
         // `last` has 4 bytes per window folded out
         const bool bad = last + 4u * kChunkWindows != a_end;
         if (__any_sync(0xffffffffu, bad) && lane == 0) report_decode_error(ws, ctl, CDMA_ERR_CORRUPT_STREAM);
@@ -380,6 +393,7 @@ cudaError_t launch_groups(const void* d_src, uint64_t src_bytes, const uint64_t*
                           uint64_t* d_ws, const LaunchCtl& ctl, cudaStream_t stream, bool src_on_device,
                           const void* d_gate) {
     const uint64_t chunks = num_chunks_of(n);
+    constexpr uint32_t kQ = Geometry<S>::kQ;
     const dim3 grid(static_cast<unsigned>((chunks + kQ - 1) / kQ));
     // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
     const bool prefetch = d_gate == nullptr && src_on_device && src_bytes >= (n * S) / 5;
