@@ -266,7 +266,10 @@ cudaError_t launch_zvc_gate_u32(const void* d_src, uint64_t src_bytes, const uin
     if (chunks == 0) return cudaSuccess;
     const dim3 grid(static_cast<unsigned>((chunks + kDecWarps - 1) / kDecWarps));
     timing_before_launch(stream);
-    zvc_decompress_kernel<uint32_t, false, true><<<grid, kDecThreads, 0, stream>>>(
+    // (the payload is asked for ahead of time under the same condition as in decompression)
+    const bool prefetch = !in_host_memory(d_src) && src_bytes >= (n * 4) / 5;
+    auto kernel = prefetch ? zvc_decompress_kernel<uint32_t, true, true> : zvc_decompress_kernel<uint32_t, false, true>;
+    kernel<<<grid, kDecThreads, 0, stream>>>(
         static_cast<const uint8_t*>(d_src), src_bytes, d_table, n, static_cast<uint32_t*>(d_dst), d_ws, ctl, chunks,
         static_cast<const uint32_t*>(d_gate));
     timing_after_launch(stream);

@@ -396,9 +396,10 @@ cudaError_t launch_groups(const void* d_src, uint64_t src_bytes, const uint64_t*
     constexpr uint32_t kQ = Geometry<S>::kQ;
     const dim3 grid(static_cast<unsigned>((chunks + kQ - 1) / kQ));
     // payload at least a fifth of the dense bytes: reading it is a real share of the traffic
-    const bool prefetch = d_gate == nullptr && src_on_device && src_bytes >= (n * S) / 5;
+    const bool prefetch = src_on_device && src_bytes >= (n * S) / 5;
     const bool bulk = src_on_device && (reinterpret_cast<uintptr_t>(d_src) & 15) == 0;
-    auto kernel = d_gate != nullptr ? (bulk ? zvc_decompress_groups_kernel<S, true, false, true>
+    auto kernel = d_gate != nullptr ? (bulk ? (prefetch ? zvc_decompress_groups_kernel<S, true, true, true>
+                                                        : zvc_decompress_groups_kernel<S, true, false, true>)
                                             : zvc_decompress_groups_kernel<S, false, false, true>)
                   : bulk ? (prefetch ? zvc_decompress_groups_kernel<S, true, true, false>
                                      : zvc_decompress_groups_kernel<S, true, false, false>)
